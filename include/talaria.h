@@ -1,0 +1,271 @@
+/*
+ * talaria.h -- C ABI of the instance-local KV substrate hot path.
+ *
+ * Four operations from the Talaria paper's memory substrate (Sec. 3.5, 4.3, 4.4):
+ *   (1) chained block hashing and prefix matching of a continuation against a
+ *       stored session stream,
+ *   (2) KV offload: gather of a session's paged KV blocks from the HBM pool
+ *       into pinned host memory (the host KV registry's checkpoint),
+ *   (3) KV restore: scatter from pinned host memory into newly allocated pool
+ *       blocks,
+ *   (4) D2D staging: copy of staged weight / KV chunks into stable-address
+ *       slots, with dirty or missing chunks reloaded from the host copy.
+ *
+ * General rules
+ *   - Every function returns a talaria_status_t (0 = OK, negative = error).
+ *     No exceptions, no aborts, no device traps.  Arguments are validated on
+ *     the host before any launch, so a bad table never reaches the GPU.
+ *   - Ownership: the caller owns all memory named in the arguments (pool,
+ *     host images, token arrays, tables, staging region, slots).  The library
+ *     owns only its context: small descriptor buffers, a device bounce buffer
+ *     for the copy-engine variant, internal streams and events.
+ *   - "HOST" / "DEVICE" beside a pointer says where it must live.  Host arrays
+ *     of tables, offsets and plans are copied before the call returns.
+ *   - Work is enqueued on the caller's CUDA stream (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and is asynchronous unless
+ *     noted.  Completion = talaria_sync() or any stream/event wait.
+ *   - A context serialises its own calls with a mutex; two calls that overlap
+ *     on the GPU must not touch the same bytes.
+ *   - GPU: sm_100a only.  There is no CPU fallback.
+ */
+#ifndef TALARIA_H_
+#define TALARIA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t talaria_status_t;
+enum {
+  TALARIA_OK = 0,
+  TALARIA_ERR_INVALID_ARG = -1,     /* null pointer, negative size, bad shape or strides  */
+  TALARIA_ERR_BAD_BLOCK_ID = -2,    /* table entry < 0 or >= num_blocks                   */
+  TALARIA_ERR_DUP_BLOCK = -3,       /* duplicate id in a restore/scatter table            */
+  TALARIA_ERR_HOST_NOT_PINNED = -4, /* host buffer is not page-locked / device-mapped     */
+  TALARIA_ERR_EXTENT = -5,          /* image or buffer smaller than the strides require   */
+  TALARIA_ERR_OVERLAP = -6,         /* stage plan: destinations overlap each other or a   */
+                                    /* source that is read                                */
+  TALARIA_ERR_CUDA = -7,            /* a CUDA call failed: see talaria_last_cuda_error    */
+  TALARIA_ERR_TIMEOUT = -8,         /* reserved: no device-side wait exists on this path  */
+  TALARIA_ERR_NO_MEMORY = -9        /* host or device allocation for the context failed   */
+};
+
+/* How offload / restore cross the host link. */
+enum {
+  TALARIA_VARIANT_AUTO = 0,     /* chosen per transfer size from the measured crossover        */
+  TALARIA_VARIANT_ZEROCOPY = 1, /* one kernel reads/writes device-mapped pinned memory         */
+  TALARIA_VARIANT_BOUNCE = 2,   /* gather kernel -> device bounce -> large copy-engine copies, */
+                                /* double-buffered on two internal streams                     */
+  TALARIA_VARIANT_RUNS = 3      /* one copy-engine copy per run of adjacent block ids          */
+};
+
+typedef struct talaria_ctx talaria_ctx;
+
+typedef struct {
+  int64_t bounce_bytes;   /* device bounce buffer PER DIRECTION (two halves); 0 = 128 MiB     */
+  int64_t dma_min_bytes;  /* AUTO: payloads >= this use BOUNCE; 0 = built-in measured value   */
+  int32_t variant;        /* TALARIA_VARIANT_*; overridden by env TALARIA_VARIANT=1|2|3       */
+  int32_t validate;       /* 0 = skip host-side table / plan validation; default 1            */
+  int32_t zc_ctas;        /* grid size of zero-copy kernels; 0 = built-in (leaves SMs free)   */
+  int32_t hbm_ctas_per_sm;/* resident CTAs per SM for HBM-bound kernels; 0 = built-in         */
+} talaria_config_t;
+
+/* Device-side paged KV pool (Sec. 4.3; descriptor fields of App. C "Attention-layout
+ * metadata": page size, dtype width, slab shape).  Plane (l, p) is one layer's K
+ * (p = 0) or V (p = 1) tensor laid out [num_blocks, kv_heads, block_tokens, head_dim];
+ * a "chunk" is one block of one plane: kv_heads*block_tokens*head_dim*elt_bytes
+ * contiguous bytes.  The addresses are stable for the life of the pool. */
+typedef struct {
+  int32_t num_layers, num_kv_heads, block_tokens, head_dim, elt_bytes;
+  int32_t num_planes;        /* 2 = paired K/V slabs (MHA); 1 = one latent slab (MLA)        */
+  int64_t num_blocks;        /* pool capacity per plane                                      */
+  void *const *plane_base;   /* HOST array [num_layers*num_planes] of DEVICE pointers        */
+} talaria_kv_layout_t;
+
+/* Image of n logical blocks outside the pool (App. C "Layer-first and page-first
+ * movement").  Chunk (l, p, i) lives at byte offset l*stride_layer + p*stride_plane
+ * + i*stride_block.  Layer-first: stride_block = C, stride_plane = n*C, stride_layer
+ * = planes*n*C.  Page-first: stride_plane = C, stride_layer = planes*C, stride_block
+ * = layers*planes*C.  Padded variants are allowed as long as the three dimensions
+ * nest without overlap; every stride and the image base must be 16-byte aligned
+ * unless the chunk size itself is not a multiple of 16. */
+typedef struct {
+  int64_t stride_layer, stride_plane, stride_block; /* bytes */
+  int64_t capacity_bytes;                           /* size of the image buffer */
+} talaria_host_layout_t;
+
+/* Result of matching one continuation against one stored stream (App. A "Prefix
+ * reuse"; Sec. 4.3 blocks keyed by cumulative prefix hash). */
+typedef struct {
+  int64_t lcp_tokens;          /* token-level longest common prefix                          */
+  int64_t matched_blocks;      /* leading full blocks whose chained hashes are equal         */
+  int64_t reusable_tokens;     /* block_tokens * min(matched_blocks, lcp_tokens/block_tokens)*/
+  int32_t hash_token_disagree; /* 1 if hashes and tokens disagree on the block count         */
+  int32_t reserved;
+} talaria_match_t;
+
+/* One entry of a staged-switch copy plan (Sec. 4.4). */
+typedef struct {
+  const void *src_dev;   /* DEVICE staged copy of the chunk; NULL = chunk was never staged   */
+  const void *src_host;  /* HOST (pinned) authoritative copy; may be NULL if never needed    */
+  void *dst_dev;         /* DEVICE stable-address slot                                       */
+  int64_t bytes;
+  int32_t chunk_id;      /* bit index into the dirty bitmap; < 0 = never dirty               */
+  int32_t reserved;
+} talaria_copy_t;
+
+/* App. D "Path classification": staged-byte coverage and dirty bytes of a switch. */
+typedef struct {
+  int64_t d2d_bytes, h2d_bytes, dirty_chunks, missing_chunks;
+} talaria_stage_stats_t;
+
+typedef struct {
+  int64_t kernel_launches;  /* kernels of this library launched since create / reset         */
+  int64_t memcpy_calls;     /* copy-engine copies enqueued (payload and descriptors)         */
+  int64_t payload_bytes;    /* KV / weight payload bytes moved                               */
+  int32_t last_variant;     /* variant the last offload / restore actually used              */
+  int32_t reserved;
+} talaria_counters_t;
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Create a context on CUDA device `device` (cfg may be NULL).  Allocates the
+ * descriptor ring, the internal streams and the bounce buffers. */
+talaria_status_t talaria_create(talaria_ctx **out, int32_t device, const talaria_config_t *cfg);
+/* Waits for the context's own streams, frees everything it owns. */
+talaria_status_t talaria_destroy(talaria_ctx *ctx);
+
+/* Page-lock and device-map an existing HOST range so offload / restore / stage
+ * may use it (the paper's "unified pinned-memory pool", Sec. 4.3).  Memory from
+ * cudaHostAlloc / torch pinned tensors needs no registration. */
+talaria_status_t talaria_host_register(talaria_ctx *ctx, void *host, size_t bytes);
+talaria_status_t talaria_host_unregister(talaria_ctx *ctx, void *host);
+
+/* ---- (1) chained block hash and prefix match ------------------------------ */
+
+/* Sec. 4.3 / App. B: cumulative hash at page (block) boundaries.  For each full
+ * block k of d_tokens:
+ *     digest_k = sum_{j<B} mix64( u32(tok[kB+j]) + G*(j+1) )        (mod 2^64)
+ *     s_k = s_{k-1}*P + digest_k,  s_{-1} = seed;   hash_k = mix64(s_k)
+ * with mix64 the SplitMix64 finaliser, G = 0x9E3779B97F4A7C15, P = 0xD1342543DE82EF95.
+ * `seed` stands for the model-name part of the key.  The partial tail block has no
+ * hash.  d_tokens: DEVICE int32[n_tokens]; d_hashes_out: DEVICE uint64[n_tokens /
+ * block_tokens].  block_tokens >= 1. */
+talaria_status_t talaria_block_hash(talaria_ctx *ctx, const int32_t *d_tokens, int64_t n_tokens,
+                                    int32_t block_tokens, uint64_t seed, uint64_t *d_hashes_out,
+                                    void *stream);
+
+/* Batched match of n_pairs continuations, each against its own session's stored
+ * stream (App. A: LCP of the new prompt and the prior prompt plus response).
+ *   d_cont_tokens / d_sess_tokens : DEVICE int32, all pairs back to back
+ *   cont_offsets / sess_offsets   : HOST int64[n_pairs+1], token offsets (CSR)
+ *   d_sess_hashes    : DEVICE uint64 or NULL.  Stored chained hashes of each
+ *                      session's full blocks, pairs back to back (pair q starts at
+ *                      sum_{r<q} floor(Ts_r/B)).  NULL = derive them from tokens.
+ *   d_cont_hashes_out: DEVICE uint64 or NULL, same CSR rule with floor(Tc_r/B).
+ *   d_results        : DEVICE talaria_match_t[n_pairs].
+ * Fields are defined as in the struct above; matched_blocks counts k <
+ * min(floor(Tc/B), floor(Ts/B)). */
+talaria_status_t talaria_prefix_match(talaria_ctx *ctx, int32_t n_pairs,
+                                      const int32_t *d_cont_tokens, const int64_t *cont_offsets,
+                                      const int32_t *d_sess_tokens, const int64_t *sess_offsets,
+                                      const uint64_t *d_sess_hashes, int32_t block_tokens,
+                                      uint64_t seed, uint64_t *d_cont_hashes_out,
+                                      talaria_match_t *d_results, void *stream);
+
+/* Same computation with every array in HOST memory (pageable or pinned): tokens
+ * are copied to the device, matched by the same kernels, and results / hashes are
+ * copied back.  Synchronous: returns after the results are in host memory. */
+talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
+                                           const int32_t *h_cont_tokens, const int64_t *cont_offsets,
+                                           const int32_t *h_sess_tokens, const int64_t *sess_offsets,
+                                           const uint64_t *h_sess_hashes, int32_t block_tokens,
+                                           uint64_t seed, uint64_t *h_cont_hashes_out,
+                                           talaria_match_t *h_results, void *stream);
+
+/* App. B "Prefix agreement": the longest leading block range on which all R
+ * ranks committed a block and hold the same chained hash.  Pure host arithmetic.
+ * committed_blocks: HOST int64[R]; hashes: HOST uint64[R][stride]. */
+int64_t talaria_prefix_agree(int32_t n_ranks, const int64_t *committed_blocks,
+                             const uint64_t *hashes, int64_t stride);
+
+/* ---- (2)/(3) block-table copies ------------------------------------------- */
+
+/* Sec. 4.3 checkpoint: host_dst[l,p,i] <- pool_{l,p}[block_table[first_block+i]]
+ * for i < n_blocks, whole chunks.  block_table: HOST int32 (at least first_block +
+ * n_blocks entries); duplicates allowed.  host_dst: HOST pinned (cudaHostAlloc,
+ * torch pinned, or talaria_host_register) image described by hl.  The pool is only
+ * read.  Errors: BAD_BLOCK_ID, EXTENT (image exceeds capacity_bytes),
+ * HOST_NOT_PINNED, INVALID_ARG. */
+talaria_status_t talaria_kv_offload(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                    const int32_t *block_table, int64_t first_block,
+                                    int64_t n_blocks, void *host_dst,
+                                    const talaria_host_layout_t *hl, void *stream);
+
+/* Sec. 4.3 restore into new device slots: pool_{l,p}[new_block_table[first_block+i]]
+ * <- host_src[l,p,i] for i < n_blocks; every other pool byte is left unchanged.
+ * Duplicate ids are rejected (DUP_BLOCK) because the result would depend on copy
+ * order. */
+talaria_status_t talaria_kv_restore(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                    const int32_t *new_block_table, int64_t first_block,
+                                    int64_t n_blocks, const void *host_src,
+                                    const talaria_host_layout_t *hl, void *stream);
+
+/* Several sessions in one call (one fused launch per variant where possible). */
+typedef struct {
+  const int32_t *block_table; /* HOST */
+  int64_t first_block, n_blocks;
+  void *host;                 /* HOST pinned image (written by offload, read by restore) */
+  talaria_host_layout_t hl;
+} talaria_kv_xfer_t;
+talaria_status_t talaria_kv_offload_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                          const talaria_kv_xfer_t *xfers, int32_t n_xfers,
+                                          void *stream);
+talaria_status_t talaria_kv_restore_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                          const talaria_kv_xfer_t *xfers, int32_t n_xfers,
+                                          void *stream);
+
+/* The same block-table gather / scatter with the image in DEVICE memory (the
+ * in-HBM leg of the bounce variant, exposed for callers that pack KV pages on
+ * the device, App. C "pack and unpack KV pages"). */
+talaria_status_t talaria_kv_gather(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                   const int32_t *block_table, int64_t first_block,
+                                   int64_t n_blocks, void *d_image,
+                                   const talaria_host_layout_t *il, void *stream);
+talaria_status_t talaria_kv_scatter(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                    const int32_t *new_block_table, int64_t first_block,
+                                    int64_t n_blocks, const void *d_image,
+                                    const talaria_host_layout_t *il, void *stream);
+
+/* ---- (4) staged switching -------------------------------------------------- */
+
+/* Sec. 4.4 gather plan: for each of the n entries, dst_dev[0..bytes) <- src_dev
+ * if the chunk is clean and present, else <- src_host (dirty: bit chunk_id of
+ * dirty_bitmap set, LSB-first bytes; missing: src_dev == NULL).  plan and
+ * dirty_bitmap are HOST arrays (bitmap may be NULL = all clean; it must cover the
+ * largest chunk_id).  src_host must be pinned where it is used.  Destinations must
+ * be pairwise disjoint and disjoint from every staged source that is read
+ * (OVERLAP).  stats (HOST, nullable) is filled before return. */
+talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                               const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
+                               void *stream);
+
+/* ---- completion, errors, counters ------------------------------------------ */
+
+/* Sec. 4.3 / App. B "Switch barrier": block the host until everything enqueued on
+ * `stream` (offloads included) has finished. */
+talaria_status_t talaria_sync(talaria_ctx *ctx, void *stream);
+
+const char *talaria_strerror(talaria_status_t status);
+/* cudaError_t value of the last failed CUDA call in this context (0 if none). */
+int32_t talaria_last_cuda_error(talaria_ctx *ctx);
+talaria_status_t talaria_get_counters(talaria_ctx *ctx, talaria_counters_t *out);
+talaria_status_t talaria_reset_counters(talaria_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TALARIA_H_ */

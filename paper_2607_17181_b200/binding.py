@@ -1,0 +1,306 @@
+"""Thin ctypes binding of libtalaria (argument marshalling only).
+
+Every method has the name of the C entry point it calls (``include/talaria.h``)
+and passes raw pointers: device memory comes from ``tensor.data_ptr()`` of torch
+tensors, host memory from pinned torch tensors or numpy arrays.  Nothing is
+computed here and there is no fallback: if the CUDA library is missing the
+import of :func:`lib` fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_CSRC = os.path.join(_HERE, "csrc")
+_INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
+LIB_PATH = os.path.join(_HERE, "libtalaria.so")
+SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "stage.cu"]
+
+OK = 0
+ERR_INVALID_ARG, ERR_BAD_BLOCK_ID, ERR_DUP_BLOCK, ERR_HOST_NOT_PINNED = -1, -2, -3, -4
+ERR_EXTENT, ERR_OVERLAP, ERR_CUDA, ERR_TIMEOUT, ERR_NO_MEMORY = -5, -6, -7, -8, -9
+VARIANT_AUTO, VARIANT_ZEROCOPY, VARIANT_BOUNCE, VARIANT_RUNS = 0, 1, 2, 3
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the CUDA sources for sm_100a into libtalaria.so (in-tree)."""
+    srcs = [os.path.join(_CSRC, s) for s in SOURCES]
+    deps = srcs + [os.path.join(_CSRC, "internal.h"), os.path.join(_INCLUDE, "talaria.h")]
+    if not force and os.path.exists(LIB_PATH) and all(
+            os.path.getmtime(LIB_PATH) >= os.path.getmtime(d) for d in deps):
+        return LIB_PATH
+    tmp = LIB_PATH + f".tmp{os.getpid()}"
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-I", _INCLUDE, "-I", _CSRC, "-o", tmp] + srcs
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
+    return LIB_PATH
+
+
+class Config(C.Structure):
+    _fields_ = [("bounce_bytes", C.c_int64), ("dma_min_bytes", C.c_int64), ("variant", C.c_int32),
+                ("validate", C.c_int32), ("zc_ctas", C.c_int32), ("hbm_ctas_per_sm", C.c_int32)]
+
+
+class KvLayout(C.Structure):
+    _fields_ = [("num_layers", C.c_int32), ("num_kv_heads", C.c_int32), ("block_tokens", C.c_int32),
+                ("head_dim", C.c_int32), ("elt_bytes", C.c_int32), ("num_planes", C.c_int32),
+                ("num_blocks", C.c_int64), ("plane_base", C.POINTER(C.c_void_p))]
+
+
+class HostLayout(C.Structure):
+    _fields_ = [("stride_layer", C.c_int64), ("stride_plane", C.c_int64), ("stride_block", C.c_int64),
+                ("capacity_bytes", C.c_int64)]
+
+
+class Match(C.Structure):
+    _fields_ = [("lcp_tokens", C.c_int64), ("matched_blocks", C.c_int64), ("reusable_tokens", C.c_int64),
+                ("hash_token_disagree", C.c_int32), ("reserved", C.c_int32)]
+
+
+MATCH_DTYPE = np.dtype([("lcp_tokens", "<i8"), ("matched_blocks", "<i8"), ("reusable_tokens", "<i8"),
+                        ("hash_token_disagree", "<i4"), ("reserved", "<i4")])
+
+
+class Copy(C.Structure):
+    _fields_ = [("src_dev", C.c_void_p), ("src_host", C.c_void_p), ("dst_dev", C.c_void_p),
+                ("bytes", C.c_int64), ("chunk_id", C.c_int32), ("reserved", C.c_int32)]
+
+
+COPY_DTYPE = np.dtype([("src_dev", "<u8"), ("src_host", "<u8"), ("dst_dev", "<u8"), ("bytes", "<i8"),
+                       ("chunk_id", "<i4"), ("reserved", "<i4")])
+
+
+class StageStats(C.Structure):
+    _fields_ = [("d2d_bytes", C.c_int64), ("h2d_bytes", C.c_int64), ("dirty_chunks", C.c_int64),
+                ("missing_chunks", C.c_int64)]
+
+
+class Counters(C.Structure):
+    _fields_ = [("kernel_launches", C.c_int64), ("memcpy_calls", C.c_int64), ("payload_bytes", C.c_int64),
+                ("last_variant", C.c_int32), ("reserved", C.c_int32)]
+
+
+class KvXfer(C.Structure):
+    _fields_ = [("block_table", C.c_void_p), ("first_block", C.c_int64), ("n_blocks", C.c_int64),
+                ("host", C.c_void_p), ("hl", HostLayout)]
+
+
+_P = C.c_void_p
+_SIGNATURES = {
+    "talaria_create": (C.c_int32, [C.POINTER(_P), C.c_int32, C.POINTER(Config)]),
+    "talaria_destroy": (C.c_int32, [_P]),
+    "talaria_host_register": (C.c_int32, [_P, _P, C.c_size_t]),
+    "talaria_host_unregister": (C.c_int32, [_P, _P]),
+    "talaria_block_hash": (C.c_int32, [_P, _P, C.c_int64, C.c_int32, C.c_uint64, _P, _P]),
+    "talaria_prefix_match": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
+    "talaria_prefix_match_host": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
+    "talaria_prefix_agree": (C.c_int64, [C.c_int32, _P, _P, C.c_int64]),
+    "talaria_kv_offload": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
+    "talaria_kv_restore": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
+    "talaria_kv_gather": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
+    "talaria_kv_scatter": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
+    "talaria_kv_offload_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
+    "talaria_kv_restore_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
+    "talaria_stage": (C.c_int32, [_P, _P, C.c_int64, _P, C.POINTER(StageStats), _P]),
+    "talaria_sync": (C.c_int32, [_P, _P]),
+    "talaria_strerror": (C.c_char_p, [C.c_int32]),
+    "talaria_last_cuda_error": (C.c_int32, [_P]),
+    "talaria_get_counters": (C.c_int32, [_P, C.POINTER(Counters)]),
+    "talaria_reset_counters": (C.c_int32, [_P]),
+}
+
+_lib = None
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built: there is no
+    CPU or PyTorch fallback for any operation."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
+        _lib = C.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            f = getattr(_lib, name)
+            f.restype, f.argtypes = res, args
+    return _lib
+
+
+class TalariaError(RuntimeError):
+    def __init__(self, status: int, what: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        msg = lib().talaria_strerror(status).decode()
+        super().__init__(f"{what}: {msg} (status {status}, cuda error {cuda_error})")
+
+
+def _ptr(x) -> Optional[int]:
+    """Raw address of a torch tensor, numpy array, int or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return x.data_ptr()  # torch tensor
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i64(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def kv_layout(shape, plane_ptrs: Sequence[int], num_blocks: int):
+    """(KvLayout, keep-alive) from a shape with the paper's descriptor fields and a
+    list of device addresses, one per (layer, plane)."""
+    n = shape.num_layers * shape.num_planes
+    assert len(plane_ptrs) == n
+    arr = (C.c_void_p * n)(*plane_ptrs)
+    kv = KvLayout(shape.num_layers, shape.num_kv_heads, shape.block_tokens, shape.head_dim,
+                  shape.elt_bytes, shape.num_planes, num_blocks, C.cast(arr, C.POINTER(C.c_void_p)))
+    return kv, arr
+
+
+def host_layout(strides, capacity_bytes: int) -> HostLayout:
+    return HostLayout(strides[0], strides[1], strides[2], capacity_bytes)
+
+
+class Talaria:
+    """One library context on one CUDA device."""
+
+    def __init__(self, device: int = 0, variant: int = VARIANT_AUTO, bounce_bytes: int = 0,
+                 dma_min_bytes: int = 0, validate: bool = True, zc_ctas: int = 0, hbm_ctas_per_sm: int = 0):
+        self._h = C.c_void_p()
+        cfg = Config(bounce_bytes, dma_min_bytes, variant, 1 if validate else 0, zc_ctas, hbm_ctas_per_sm)
+        rc = lib().talaria_create(C.byref(self._h), device, C.byref(cfg))
+        if rc != OK:
+            self._h = C.c_void_p()
+            raise TalariaError(rc, "talaria_create")
+
+    def _check(self, rc: int, what: str):
+        if rc != OK:
+            raise TalariaError(rc, what, lib().talaria_last_cuda_error(self._h))
+
+    def destroy(self):
+        if self._h:
+            lib().talaria_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    # -- pinned memory ------------------------------------------------------
+    def host_register(self, arr: np.ndarray):
+        self._check(lib().talaria_host_register(self._h, arr.ctypes.data, arr.nbytes), "talaria_host_register")
+
+    def host_unregister(self, arr: np.ndarray):
+        self._check(lib().talaria_host_unregister(self._h, arr.ctypes.data), "talaria_host_unregister")
+
+    # -- (1) hashing and matching ------------------------------------------
+    def block_hash(self, d_tokens, n_tokens: int, block_tokens: int, seed: int, d_hashes_out, stream=None):
+        self._check(lib().talaria_block_hash(self._h, _ptr(d_tokens), n_tokens, block_tokens,
+                                             C.c_uint64(seed), _ptr(d_hashes_out), _stream_ptr(stream)),
+                    "talaria_block_hash")
+
+    def prefix_match(self, n_pairs: int, d_cont_tokens, cont_offsets, d_sess_tokens, sess_offsets,
+                     d_sess_hashes, block_tokens: int, seed: int, d_cont_hashes_out, d_results, stream=None):
+        co, so = _i64(cont_offsets), _i64(sess_offsets)
+        self._check(lib().talaria_prefix_match(self._h, n_pairs, _ptr(d_cont_tokens), _ptr(co),
+                                               _ptr(d_sess_tokens), _ptr(so), _ptr(d_sess_hashes),
+                                               block_tokens, C.c_uint64(seed), _ptr(d_cont_hashes_out),
+                                               _ptr(d_results), _stream_ptr(stream)), "talaria_prefix_match")
+
+    def prefix_match_host(self, n_pairs: int, h_cont_tokens, cont_offsets, h_sess_tokens, sess_offsets,
+                          h_sess_hashes, block_tokens: int, seed: int, h_cont_hashes_out, h_results,
+                          stream=None):
+        co, so = _i64(cont_offsets), _i64(sess_offsets)
+        self._check(lib().talaria_prefix_match_host(self._h, n_pairs, _ptr(h_cont_tokens), _ptr(co),
+                                                    _ptr(h_sess_tokens), _ptr(so), _ptr(h_sess_hashes),
+                                                    block_tokens, C.c_uint64(seed), _ptr(h_cont_hashes_out),
+                                                    _ptr(h_results), _stream_ptr(stream)),
+                    "talaria_prefix_match_host")
+
+    @staticmethod
+    def prefix_agree(committed_blocks, hashes: np.ndarray) -> int:
+        cb = _i64(committed_blocks)
+        h = np.ascontiguousarray(hashes, dtype=np.uint64)
+        assert h.ndim == 2 and h.shape[0] == cb.size
+        return int(lib().talaria_prefix_agree(cb.size, _ptr(cb), _ptr(h), h.shape[1]))
+
+    # -- (2)/(3) block-table copies ----------------------------------------
+    def _kv(self, fn, what, kv, table, first, n, image, hl, stream):
+        bt = _i32(table)
+        self._check(fn(self._h, C.byref(kv), _ptr(bt), first, n, _ptr(image), C.byref(hl), _stream_ptr(stream)), what)
+
+    def kv_offload(self, kv, block_table, first_block, n_blocks, host_dst, hl, stream=None):
+        self._kv(lib().talaria_kv_offload, "talaria_kv_offload", kv, block_table, first_block, n_blocks, host_dst, hl, stream)
+
+    def kv_restore(self, kv, new_block_table, first_block, n_blocks, host_src, hl, stream=None):
+        self._kv(lib().talaria_kv_restore, "talaria_kv_restore", kv, new_block_table, first_block, n_blocks, host_src, hl, stream)
+
+    def kv_gather(self, kv, block_table, first_block, n_blocks, d_image, il, stream=None):
+        self._kv(lib().talaria_kv_gather, "talaria_kv_gather", kv, block_table, first_block, n_blocks, d_image, il, stream)
+
+    def kv_scatter(self, kv, new_block_table, first_block, n_blocks, d_image, il, stream=None):
+        self._kv(lib().talaria_kv_scatter, "talaria_kv_scatter", kv, new_block_table, first_block, n_blocks, d_image, il, stream)
+
+    def _batch(self, fn, what, kv, xfers, stream):
+        """xfers: sequence of (block_table, first_block, n_blocks, host_image, HostLayout)."""
+        arr = (KvXfer * max(len(xfers), 1))()
+        keep = []
+        for k, (bt, first, n, img, hl) in enumerate(xfers):
+            bt = _i32(bt)
+            keep.append(bt)
+            arr[k] = KvXfer(_ptr(bt), first, n, _ptr(img), hl)
+        self._check(fn(self._h, C.byref(kv), arr, len(xfers), _stream_ptr(stream)), what)
+
+    def kv_offload_batch(self, kv, xfers, stream=None):
+        self._batch(lib().talaria_kv_offload_batch, "talaria_kv_offload_batch", kv, xfers, stream)
+
+    def kv_restore_batch(self, kv, xfers, stream=None):
+        self._batch(lib().talaria_kv_restore_batch, "talaria_kv_restore_batch", kv, xfers, stream)
+
+    # -- (4) staging --------------------------------------------------------
+    def stage(self, plan: np.ndarray, dirty_bitmap: Optional[np.ndarray] = None, stream=None) -> StageStats:
+        """plan: numpy structured array of COPY_DTYPE (raw addresses)."""
+        plan = np.ascontiguousarray(plan, dtype=COPY_DTYPE)
+        bm = None if dirty_bitmap is None else np.ascontiguousarray(dirty_bitmap, dtype=np.uint8)
+        st = StageStats()
+        self._check(lib().talaria_stage(self._h, _ptr(plan), plan.size, _ptr(bm), C.byref(st),
+                                        _stream_ptr(stream)), "talaria_stage")
+        return st
+
+    # -- completion and counters ---------------------------------------------
+    def sync(self, stream=None):
+        self._check(lib().talaria_sync(self._h, _stream_ptr(stream)), "talaria_sync")
+
+    def get_counters(self) -> Counters:
+        c = Counters()
+        self._check(lib().talaria_get_counters(self._h, C.byref(c)), "talaria_get_counters")
+        return c
+
+    def reset_counters(self):
+        self._check(lib().talaria_reset_counters(self._h), "talaria_reset_counters")

@@ -1,0 +1,270 @@
+// Context, error handling, descriptor ring, pinned-memory registration.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+namespace tal {
+
+talaria_status_t cuda_fail(talaria_ctx *ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda_error = (int32_t)e;
+  (void)cudaGetLastError();  // clear the sticky-free error so later calls start clean
+  return TALARIA_ERR_CUDA;
+}
+
+talaria_status_t acquire_slot(talaria_ctx *ctx, size_t bytes, DescSlot **out) {
+  DescSlot &s = ctx->ring[ctx->ring_next];
+  ctx->ring_next = (ctx->ring_next + 1) % kRing;
+  if (s.used) {
+    TAL_CUDA(ctx, cudaEventSynchronize(s.ev));
+    s.used = false;
+  }
+  if (s.cap < bytes) {
+    size_t cap = std::max<size_t>(bytes + bytes / 2, 64 << 10);
+    if (s.h) cudaFreeHost(s.h);
+    if (s.d) cudaFree(s.d);
+    s.h = s.d = nullptr;
+    s.cap = 0;
+    TAL_CUDA(ctx, cudaHostAlloc((void **)&s.h, cap, cudaHostAllocDefault));
+    TAL_CUDA(ctx, cudaMalloc((void **)&s.d, cap));
+    s.cap = cap;
+  }
+  *out = &s;
+  return TALARIA_OK;
+}
+
+talaria_status_t upload_slot(talaria_ctx *ctx, DescSlot *slot, size_t bytes, cudaStream_t stream) {
+  if (bytes == 0) return TALARIA_OK;
+  TAL_CUDA(ctx, cudaMemcpyAsync(slot->d, slot->h, bytes, cudaMemcpyHostToDevice, stream));
+  ctx->counters.memcpy_calls++;
+  return TALARIA_OK;
+}
+
+talaria_status_t release_slot(talaria_ctx *ctx, DescSlot *slot, cudaStream_t stream) {
+  TAL_CUDA(ctx, cudaEventRecord(slot->ev, stream));
+  slot->used = true;
+  return TALARIA_OK;
+}
+
+talaria_status_t grow(talaria_ctx *ctx, DevBuf *b, size_t bytes) {
+  if (b->cap >= bytes) return TALARIA_OK;
+  size_t cap = std::max<size_t>(bytes + bytes / 4, 1 << 20);
+  if (b->p) {
+    // cudaFree waits for the device, so nothing still reads the old buffer
+    TAL_CUDA(ctx, cudaFree(b->p));
+    b->p = nullptr;
+    b->cap = 0;
+  }
+  cudaError_t e = cudaMalloc((void **)&b->p, cap);
+  if (e == cudaErrorMemoryAllocation) {
+    (void)cudaGetLastError();
+    return TALARIA_ERR_NO_MEMORY;
+  }
+  TAL_CUDA(ctx, e);
+  b->cap = cap;
+  return TALARIA_OK;
+}
+
+talaria_status_t mapped_pointer(talaria_ctx *ctx, const void *host, void **dev_alias) {
+  cudaPointerAttributes a{};
+  cudaError_t e = cudaPointerGetAttributes(&a, host);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return TALARIA_ERR_HOST_NOT_PINNED;
+  }
+  if (a.type != cudaMemoryTypeHost || a.devicePointer == nullptr) return TALARIA_ERR_HOST_NOT_PINNED;
+  (void)ctx;
+  *dev_alias = a.devicePointer;
+  return TALARIA_OK;
+}
+
+talaria_status_t require_device_pointer(talaria_ctx *ctx, const void *p) {
+  cudaPointerAttributes a{};
+  cudaError_t e = cudaPointerGetAttributes(&a, p);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return TALARIA_ERR_INVALID_ARG;
+  }
+  if (a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged) {
+    if (a.type == cudaMemoryTypeDevice && a.device != ctx->device) return TALARIA_ERR_INVALID_ARG;
+    return TALARIA_OK;
+  }
+  return TALARIA_ERR_INVALID_ARG;
+}
+
+int hbm_grid(const talaria_ctx *ctx, int threads_per_cta) {
+  int per_sm = ctx->cfg.hbm_ctas_per_sm > 0 ? ctx->cfg.hbm_ctas_per_sm : std::max(1, 2048 / threads_per_cta);
+  return ctx->sm_count * per_sm;
+}
+
+}  // namespace tal
+
+using namespace tal;
+
+static void destroy_impl(talaria_ctx *ctx) {
+  for (auto &ln : ctx->lane) {
+    for (int j = 0; j < 2; ++j) {
+      if (ln.s[j]) {
+        cudaStreamSynchronize(ln.s[j]);
+        cudaStreamDestroy(ln.s[j]);
+      }
+      if (ln.done[j]) cudaEventDestroy(ln.done[j]);
+    }
+    if (ln.fork) cudaEventDestroy(ln.fork);
+    if (ln.buf) cudaFree(ln.buf);
+  }
+  for (auto &s : ctx->ring) {
+    if (s.used) cudaEventSynchronize(s.ev);
+    if (s.ev) cudaEventDestroy(s.ev);
+    if (s.h) cudaFreeHost(s.h);
+    if (s.d) cudaFree(s.d);
+  }
+  if (ctx->prefix_scratch.p) cudaFree(ctx->prefix_scratch.p);
+  if (ctx->host_tok.p) cudaFree(ctx->host_tok.p);
+  for (auto &r : ctx->registered) cudaHostUnregister(r.first);
+  (void)cudaGetLastError();
+  delete ctx;
+}
+
+extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, const talaria_config_t *cfg) {
+  if (!out) return TALARIA_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    (void)cudaGetLastError();
+    return TALARIA_ERR_CUDA;
+  }
+  talaria_ctx *ctx = new (std::nothrow) talaria_ctx();
+  if (!ctx) return TALARIA_ERR_NO_MEMORY;
+  ctx->device = device;
+  if (cfg) ctx->cfg = *cfg;
+  if (!cfg) ctx->cfg.validate = 1;
+  if (ctx->cfg.bounce_bytes <= 0) ctx->cfg.bounce_bytes = 128ll << 20;
+  if (ctx->cfg.bounce_bytes < (1 << 20)) ctx->cfg.bounce_bytes = 1 << 20;
+  if (const char *v = getenv("TALARIA_VARIANT")) {
+    int x = atoi(v);
+    if (x >= TALARIA_VARIANT_AUTO && x <= TALARIA_VARIANT_RUNS) ctx->cfg.variant = x;
+  }
+  if (ctx->cfg.variant < TALARIA_VARIANT_AUTO || ctx->cfg.variant > TALARIA_VARIANT_RUNS) {
+    delete ctx;
+    return TALARIA_ERR_INVALID_ARG;
+  }
+  DeviceGuard g(device);
+  talaria_status_t st = [&]() -> talaria_status_t {
+    if (!g.ok) return TALARIA_ERR_CUDA;
+    cudaDeviceProp prop{};
+    TAL_CUDA(ctx, cudaGetDeviceProperties(&prop, device));
+    ctx->sm_count = prop.multiProcessorCount;
+    for (auto &s : ctx->ring) TAL_CUDA(ctx, cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming));
+    for (auto &ln : ctx->lane) {
+      for (int j = 0; j < 2; ++j) {
+        TAL_CUDA(ctx, cudaStreamCreateWithFlags(&ln.s[j], cudaStreamNonBlocking));
+        TAL_CUDA(ctx, cudaEventCreateWithFlags(&ln.done[j], cudaEventDisableTiming));
+      }
+      TAL_CUDA(ctx, cudaEventCreateWithFlags(&ln.fork, cudaEventDisableTiming));
+      ln.half = ((size_t)ctx->cfg.bounce_bytes / 2) & ~(size_t)255;
+      cudaError_t e = cudaMalloc((void **)&ln.buf, ln.half * 2);
+      if (e == cudaErrorMemoryAllocation) {
+        (void)cudaGetLastError();
+        return TALARIA_ERR_NO_MEMORY;
+      }
+      TAL_CUDA(ctx, e);
+    }
+    return TALARIA_OK;
+  }();
+  if (st != TALARIA_OK) {
+    destroy_impl(ctx);
+    return st;
+  }
+  *out = ctx;
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_destroy(talaria_ctx *ctx) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  destroy_impl(ctx);
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_host_register(talaria_ctx *ctx, void *host, size_t bytes) {
+  if (!ctx || !host || bytes == 0) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  DeviceGuard g(ctx->device);
+  TAL_CUDA(ctx, cudaHostRegister(host, bytes, cudaHostRegisterMapped | cudaHostRegisterPortable));
+  ctx->registered.emplace_back((char *)host, bytes);
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_host_unregister(talaria_ctx *ctx, void *host) {
+  if (!ctx || !host) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  DeviceGuard g(ctx->device);
+  for (size_t k = 0; k < ctx->registered.size(); ++k) {
+    if (ctx->registered[k].first == (char *)host) {
+      TAL_CUDA(ctx, cudaHostUnregister(host));
+      ctx->registered.erase(ctx->registered.begin() + k);
+      return TALARIA_OK;
+    }
+  }
+  return TALARIA_ERR_INVALID_ARG;
+}
+
+extern "C" talaria_status_t talaria_sync(talaria_ctx *ctx, void *stream) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  TAL_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+  return TALARIA_OK;
+}
+
+extern "C" const char *talaria_strerror(talaria_status_t s) {
+  switch (s) {
+    case TALARIA_OK: return "ok";
+    case TALARIA_ERR_INVALID_ARG: return "invalid argument";
+    case TALARIA_ERR_BAD_BLOCK_ID: return "block id out of range";
+    case TALARIA_ERR_DUP_BLOCK: return "duplicate block id in a restore table";
+    case TALARIA_ERR_HOST_NOT_PINNED: return "host buffer is not pinned / device-mapped";
+    case TALARIA_ERR_EXTENT: return "buffer smaller than the layout requires";
+    case TALARIA_ERR_OVERLAP: return "stage plan ranges overlap";
+    case TALARIA_ERR_CUDA: return "CUDA call failed (see talaria_last_cuda_error)";
+    case TALARIA_ERR_TIMEOUT: return "timeout";
+    case TALARIA_ERR_NO_MEMORY: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+extern "C" int32_t talaria_last_cuda_error(talaria_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+extern "C" talaria_status_t talaria_get_counters(talaria_ctx *ctx, talaria_counters_t *out) {
+  if (!ctx || !out) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  *out = ctx->counters;
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_reset_counters(talaria_ctx *ctx) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  int32_t v = ctx->counters.last_variant;
+  ctx->counters = talaria_counters_t{};
+  ctx->counters.last_variant = v;
+  return TALARIA_OK;
+}
+
+extern "C" int64_t talaria_prefix_agree(int32_t n_ranks, const int64_t *committed_blocks,
+                                        const uint64_t *hashes, int64_t stride) {
+  if (n_ranks <= 0 || !committed_blocks) return 0;
+  int64_t agreed = committed_blocks[0];
+  for (int32_t r = 1; r < n_ranks; ++r) agreed = std::min(agreed, committed_blocks[r]);
+  if (agreed <= 0 || !hashes) return 0;
+  // every rank is compared with rank 0; the first column where any differs ends the prefix
+  for (int32_t r = 1; r < n_ranks; ++r) {
+    const uint64_t *a = hashes, *b = hashes + (int64_t)r * stride;
+    int64_t k = 0;
+    while (k < agreed && a[k] == b[k]) ++k;
+    agreed = k;
+  }
+  return agreed;
+}

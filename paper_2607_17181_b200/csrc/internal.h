@@ -1,0 +1,102 @@
+// Internal declarations shared by the CUDA sources of libtalaria (not installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <mutex>
+#include <utility>
+#include <vector>
+
+#include "talaria.h"
+
+namespace tal {
+
+constexpr int kRing = 8;              // descriptor slots in flight
+constexpr int kLanes = 2;             // 0: offload (device->host), 1: restore (host->device)
+
+struct DescSlot {
+  char *h = nullptr;                  // pinned staging
+  char *d = nullptr;                  // device copy
+  size_t cap = 0;
+  cudaEvent_t ev = nullptr;           // recorded after the last consumer was enqueued
+  bool used = false;
+};
+
+struct BounceLane {
+  cudaStream_t s[2] = {nullptr, nullptr};
+  cudaEvent_t done[2] = {nullptr, nullptr};
+  cudaEvent_t fork = nullptr;
+  char *buf = nullptr;                // two halves of `half` bytes
+  size_t half = 0;
+};
+
+struct DevBuf {                       // growable device scratch
+  char *p = nullptr;
+  size_t cap = 0;
+};
+
+}  // namespace tal
+
+struct talaria_ctx {
+  int device = 0;
+  int sm_count = 0;
+  talaria_config_t cfg{};
+  std::mutex mu;
+  tal::DescSlot ring[tal::kRing];
+  int ring_next = 0;
+  tal::BounceLane lane[tal::kLanes];
+  tal::DevBuf prefix_scratch;         // digests + per-tile mismatch positions
+  tal::DevBuf host_tok;               // device copies for talaria_prefix_match_host
+  std::vector<std::pair<char *, size_t>> registered;
+  std::vector<uint64_t> dup_bits;     // restore-table duplicate check
+  int32_t last_cuda_error = 0;
+  talaria_counters_t counters{};
+};
+
+namespace tal {
+
+// Records the CUDA error in the context and maps it to TALARIA_ERR_CUDA.
+talaria_status_t cuda_fail(talaria_ctx *ctx, cudaError_t e);
+
+#define TAL_CUDA(ctx, call)                                   \
+  do {                                                        \
+    cudaError_t e__ = (call);                                 \
+    if (e__ != cudaSuccess) return tal::cuda_fail((ctx), e__);\
+  } while (0)
+
+#define TAL_TRY(expr)                                         \
+  do {                                                        \
+    talaria_status_t s__ = (expr);                            \
+    if (s__ != TALARIA_OK) return s__;                        \
+  } while (0)
+
+// RAII: make the context's device current for the duration of a call.
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess) ok = true;
+  }
+  ~DeviceGuard() {
+    if (ok && prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+// Descriptor ring: a pinned + device buffer pair of at least `bytes`, free to
+// overwrite (its previous consumers have finished).
+talaria_status_t acquire_slot(talaria_ctx *ctx, size_t bytes, DescSlot **out);
+// Uploads the first `bytes` of the slot on `stream`.
+talaria_status_t upload_slot(talaria_ctx *ctx, DescSlot *slot, size_t bytes, cudaStream_t stream);
+// Marks the slot busy until everything enqueued on `stream` so far is done.
+talaria_status_t release_slot(talaria_ctx *ctx, DescSlot *slot, cudaStream_t stream);
+
+talaria_status_t grow(talaria_ctx *ctx, DevBuf *b, size_t bytes);
+
+// Device-visible alias of a pinned host range, or HOST_NOT_PINNED.
+talaria_status_t mapped_pointer(talaria_ctx *ctx, const void *host, void **dev_alias);
+// OK if `p` is device memory of this context's device.
+talaria_status_t require_device_pointer(talaria_ctx *ctx, const void *p);
+
+// Grid size for kernels that should fill the GPU (HBM-bound work).
+int hbm_grid(const talaria_ctx *ctx, int threads_per_cta);
+
+}  // namespace tal

@@ -1,0 +1,462 @@
+// Block-table copies between the paged KV pool and an image of logical blocks:
+// KV offload (pool -> pinned host), KV restore (pinned host -> new pool blocks)
+// and the in-HBM gather / scatter (Sec. 4.3; App. C layer-first / page-first).
+//
+// One kernel serves every case.  The image is enumerated in ITS OWN memory order
+// (fastest-varying dimension first), so the image side of the copy is a single
+// sequential stream -- full 128-byte lines on the host link -- while the pool side
+// jumps from chunk to chunk as the block table says.  Each warp moves 4 KiB per
+// step with eight 16-byte accesses per lane in flight.
+#include <algorithm>
+#include <cstring>
+
+#include "internal.h"
+
+namespace tal {
+
+struct ImgOrder {
+  // linear chunk index w = (d2*e1 + d1)*e0 + d0, dimension 0 innermost in the image
+  int64_t e0, e1;
+  int32_t pos_l, pos_p, pos_i;  // which digit (0,1,2) holds layer / plane / block (host use)
+  int32_t lp_coef[3];           // plane index l*P + p = sum_k d_k * lp_coef[k]
+  int32_t i_coef[3];            // logical block i   = sum_k d_k * i_coef[k]
+};
+
+struct KvCopyParams {
+  const void *const *plane_base;  // DEVICE [L*P]
+  const int32_t *table;           // DEVICE [n], already offset to first_block
+  char *img;                      // image base as seen from the device
+  int64_t sd[3];                  // image stride of digit 0, 1, 2 (bytes)
+  int64_t chunk_bytes;
+  int64_t w0, w1;                 // chunks [w0, w1) of the image order
+  int32_t P;
+  ImgOrder ord;
+};
+
+constexpr int kPart = 4096;       // bytes one warp moves per step (vector path)
+
+__device__ __forceinline__ void decode_chunk(const KvCopyParams &p, int64_t w, int64_t &lp, int64_t &i,
+                                             int64_t &img_off) {
+  const int64_t t = w / p.ord.e0;
+  const int64_t d0 = w - t * p.ord.e0;
+  const int64_t d2 = t / p.ord.e1;
+  const int64_t d1 = t - d2 * p.ord.e1;
+  lp = d0 * p.ord.lp_coef[0] + d1 * p.ord.lp_coef[1] + d2 * p.ord.lp_coef[2];
+  i = d0 * p.ord.i_coef[0] + d1 * p.ord.i_coef[1] + d2 * p.ord.i_coef[2];
+  img_off = d0 * p.sd[0] + d1 * p.sd[1] + d2 * p.sd[2];
+}
+
+// TO_IMAGE: pool -> image (offload / gather); else image -> pool (restore / scatter).
+template <bool TO_IMAGE>
+__global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant__ KvCopyParams p) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int64_t parts = (p.chunk_bytes + kPart - 1) / kPart;
+  const int64_t units = (p.w1 - p.w0) * parts;
+  for (int64_t u = warp; u < units; u += nwarps) {
+    int64_t c = u / parts;
+    int64_t part = u - c * parts;
+    int64_t lp, i, img_off;
+    decode_chunk(p, p.w0 + c, lp, i, img_off);
+    int64_t blk = p.table[i];
+    char *pool = (char *)p.plane_base[lp] + blk * p.chunk_bytes + part * kPart;
+    char *img = p.img + img_off + part * kPart;
+    const int4 *src = (const int4 *)(TO_IMAGE ? pool : img);
+    int4 *dst = (int4 *)(TO_IMAGE ? img : pool);
+    int64_t left = p.chunk_bytes - part * kPart;
+    if (left >= kPart) {
+      int4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldcs(src + lane + k * 32);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) __stcs(dst + lane + k * 32, v[k]);
+    } else {
+      int n16 = (int)(left >> 4);
+      for (int k = lane; k < n16; k += 32) __stcs(dst + k, __ldcs(src + k));
+    }
+  }
+}
+
+// Any chunk size / alignment: plain byte copies (odd shapes only).
+template <bool TO_IMAGE>
+__global__ void __launch_bounds__(256) kv_copy_byte_kernel(const __grid_constant__ KvCopyParams p) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t c = warp; c < p.w1 - p.w0; c += nwarps) {
+    int64_t lp, i, img_off;
+    decode_chunk(p, p.w0 + c, lp, i, img_off);
+    int64_t blk = p.table[i];
+    char *pool = (char *)p.plane_base[lp] + blk * p.chunk_bytes;
+    char *img = p.img + img_off;
+    const char *src = TO_IMAGE ? pool : img;
+    char *dst = TO_IMAGE ? img : pool;
+    for (int64_t k = lane; k < p.chunk_bytes; k += 32) dst[k] = src[k];
+  }
+}
+
+// ---------------------------------------------------------------------------
+
+struct Dim {
+  int64_t extent, stride;
+  int which;  // 0 layer, 1 plane, 2 block
+};
+
+struct Plan {
+  int64_t L, P, n, C, chunks;
+  ImgOrder ord;
+  int64_t run_chunks;  // chunks that are contiguous in the image, aligned in w
+  bool vec;            // 16-byte path usable
+};
+
+static talaria_status_t make_plan(const talaria_kv_layout_t *kv, int64_t n, const void *img,
+                                  const talaria_host_layout_t *hl, Plan *out) {
+  if (kv->num_layers <= 0 || kv->num_kv_heads <= 0 || kv->block_tokens <= 0 || kv->head_dim <= 0 ||
+      kv->elt_bytes <= 0 || kv->num_planes <= 0 || kv->num_blocks <= 0 || !kv->plane_base)
+    return TALARIA_ERR_INVALID_ARG;
+  Plan pl{};
+  pl.L = kv->num_layers;
+  pl.P = kv->num_planes;
+  pl.n = n;
+  pl.C = (int64_t)kv->num_kv_heads * kv->block_tokens * kv->head_dim * kv->elt_bytes;
+  pl.chunks = pl.L * pl.P * n;
+  if (hl->stride_layer < 0 || hl->stride_plane < 0 || hl->stride_block < 0 || hl->capacity_bytes < 0)
+    return TALARIA_ERR_INVALID_ARG;
+  Dim d[3] = {{pl.L, hl->stride_layer, 0}, {pl.P, hl->stride_plane, 1}, {n, hl->stride_block, 2}};
+  // innermost first; dimensions of extent 1 have no meaningful stride: keep them innermost
+  std::stable_sort(d, d + 3, [](const Dim &a, const Dim &b) {
+    bool a1 = a.extent == 1, b1 = b.extent == 1;
+    if (a1 != b1) return a1;
+    if (a1 && b1) return false;
+    return a.stride < b.stride;
+  });
+  // the three dimensions must nest without overlap
+  int64_t span = pl.C;
+  for (int k = 0; k < 3; ++k) {
+    if (d[k].extent == 1) continue;
+    if (d[k].stride < span) return TALARIA_ERR_INVALID_ARG;
+    span = d[k].stride * (d[k].extent - 1) + span;
+  }
+  if (span > hl->capacity_bytes) return TALARIA_ERR_EXTENT;
+  pl.ord.e0 = d[0].extent;
+  pl.ord.e1 = d[1].extent;
+  for (int k = 0; k < 3; ++k) {
+    pl.ord.lp_coef[k] = 0;
+    pl.ord.i_coef[k] = 0;
+    if (d[k].which == 0) { pl.ord.pos_l = k; pl.ord.lp_coef[k] = (int32_t)pl.P; }
+    if (d[k].which == 1) { pl.ord.pos_p = k; pl.ord.lp_coef[k] = 1; }
+    if (d[k].which == 2) { pl.ord.pos_i = k; pl.ord.i_coef[k] = 1; }
+  }
+  int64_t run = 1, bytes = pl.C;
+  for (int k = 0; k < 3; ++k) {
+    if (d[k].extent != 1 && d[k].stride != bytes) break;
+    run *= d[k].extent;
+    bytes *= d[k].extent;
+  }
+  pl.run_chunks = run;
+  bool aligned = (pl.C % 16 == 0) && (((uintptr_t)img) % 16 == 0);
+  for (int k = 0; k < 3; ++k)
+    if (d[k].extent != 1 && d[k].stride % 16 != 0) aligned = false;
+  for (int64_t k = 0; k < pl.L * pl.P; ++k) {
+    if (!kv->plane_base[k]) return TALARIA_ERR_INVALID_ARG;
+    if (((uintptr_t)kv->plane_base[k]) % 16 != 0) aligned = false;
+  }
+  pl.vec = aligned;
+  *out = pl;
+  return TALARIA_OK;
+}
+
+static int64_t image_offset(const Plan &pl, const talaria_host_layout_t *hl, int64_t w) {
+  int64_t d[3];
+  int64_t t = w / pl.ord.e0;
+  d[0] = w - t * pl.ord.e0;
+  d[2] = t / pl.ord.e1;
+  d[1] = t - d[2] * pl.ord.e1;
+  return d[pl.ord.pos_l] * hl->stride_layer + d[pl.ord.pos_p] * hl->stride_plane +
+         d[pl.ord.pos_i] * hl->stride_block;
+}
+
+static talaria_status_t validate_table(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const int32_t *bt,
+                                       int64_t n, bool reject_dups) {
+  if (!ctx->cfg.validate) return TALARIA_OK;
+  const int64_t nb = kv->num_blocks;
+  for (int64_t i = 0; i < n; ++i)
+    if (bt[i] < 0 || (int64_t)bt[i] >= nb) return TALARIA_ERR_BAD_BLOCK_ID;
+  if (reject_dups) {
+    size_t words = (size_t)((nb + 63) / 64);
+    ctx->dup_bits.assign(words, 0);
+    for (int64_t i = 0; i < n; ++i) {
+      uint64_t bit = 1ull << (bt[i] & 63);
+      uint64_t &w = ctx->dup_bits[(size_t)bt[i] >> 6];
+      if (w & bit) return TALARIA_ERR_DUP_BLOCK;
+      w |= bit;
+    }
+  }
+  return TALARIA_OK;
+}
+
+template <bool TO_IMAGE>
+static talaria_status_t launch_copy(talaria_ctx *ctx, const KvCopyParams &p, bool vec, int grid_cap,
+                                    cudaStream_t stream) {
+  if (p.w1 <= p.w0) return TALARIA_OK;
+  if (vec) {
+    const int threads = 512;
+    int64_t parts = (p.chunk_bytes + kPart - 1) / kPart;
+    int64_t warps = (p.w1 - p.w0) * parts;
+    int64_t need = (warps + threads / 32 - 1) / (threads / 32);
+    int grid = (int)std::max<int64_t>(1, std::min<int64_t>(need, grid_cap));
+    kv_copy_vec_kernel<TO_IMAGE><<<grid, threads, 0, stream>>>(p);
+  } else {
+    const int threads = 256;
+    int64_t need = ((p.w1 - p.w0) + threads / 32 - 1) / (threads / 32);
+    int grid = (int)std::max<int64_t>(1, std::min<int64_t>(need, grid_cap));
+    kv_copy_byte_kernel<TO_IMAGE><<<grid, threads, 0, stream>>>(p);
+  }
+  TAL_CUDA(ctx, cudaGetLastError());
+  ctx->counters.kernel_launches++;
+  return TALARIA_OK;
+}
+
+static talaria_status_t launch_dir(talaria_ctx *ctx, bool to_image, const KvCopyParams &p, bool vec,
+                                   int grid_cap, cudaStream_t stream) {
+  return to_image ? launch_copy<true>(ctx, p, vec, grid_cap, stream)
+                  : launch_copy<false>(ctx, p, vec, grid_cap, stream);
+}
+
+static void set_image_strides(KvCopyParams &p, const ImgOrder &o, int64_t sL, int64_t sP, int64_t sI) {
+  p.sd[o.pos_l] = sL;
+  p.sd[o.pos_p] = sP;
+  p.sd[o.pos_i] = sI;
+}
+
+static int zc_grid(const talaria_ctx *ctx) { return ctx->cfg.zc_ctas > 0 ? ctx->cfg.zc_ctas : 32; }
+
+// Number of runs of adjacent ids in a table (bt[i+1] == bt[i]+1 continues a run).
+static int64_t count_id_runs(const int32_t *bt, int64_t n) {
+  int64_t runs = n > 0 ? 1 : 0;
+  for (int64_t i = 1; i < n; ++i)
+    if (bt[i] != bt[i - 1] + 1) ++runs;
+  return runs;
+}
+
+// to_image: offload / gather; img_on_device: the image is device memory (gather / scatter).
+static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const int32_t *table,
+                                    int64_t first, int64_t n, void *img, const talaria_host_layout_t *hl,
+                                    cudaStream_t stream, bool to_image, bool img_on_device) {
+  if (!kv || !hl || first < 0 || n < 0) return TALARIA_ERR_INVALID_ARG;
+  if (n == 0) return TALARIA_OK;
+  if (!table || !img) return TALARIA_ERR_INVALID_ARG;
+  Plan pl;
+  TAL_TRY(make_plan(kv, n, img, hl, &pl));
+  const int32_t *bt = table + first;
+  TAL_TRY(validate_table(ctx, kv, bt, n, /*reject_dups=*/!to_image));
+
+  void *img_dev = img;
+  if (img_on_device) {
+    TAL_TRY(require_device_pointer(ctx, img));
+  } else {
+    TAL_TRY(mapped_pointer(ctx, img, &img_dev));
+    if (((uintptr_t)img_dev) % 16 != 0) pl.vec = false;
+  }
+
+  // descriptor: plane pointers, then the table slice
+  const size_t ptr_bytes = (size_t)(pl.L * pl.P) * sizeof(void *);
+  const size_t desc_bytes = ptr_bytes + (size_t)n * sizeof(int32_t);
+  DescSlot *slot;
+  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+  memcpy(slot->h, kv->plane_base, ptr_bytes);
+  memcpy(slot->h + ptr_bytes, bt, (size_t)n * sizeof(int32_t));
+  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+
+  KvCopyParams p{};
+  p.plane_base = (const void *const *)slot->d;
+  p.table = (const int32_t *)(slot->d + ptr_bytes);
+  p.chunk_bytes = pl.C;
+  p.P = (int32_t)pl.P;
+  p.ord = pl.ord;
+
+  const int64_t payload = pl.chunks * pl.C;
+  ctx->counters.payload_bytes += payload;
+
+  if (img_on_device) {
+    p.img = (char *)img_dev;
+    set_image_strides(p, pl.ord, hl->stride_layer, hl->stride_plane, hl->stride_block);
+    p.w0 = 0; p.w1 = pl.chunks;
+    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, hbm_grid(ctx, 512), stream));
+    return release_slot(ctx, slot, stream);
+  }
+
+  // ---- choose how to cross the host link --------------------------------
+  BounceLane &ln = ctx->lane[to_image ? 0 : 1];
+  const int64_t dma_min = ctx->cfg.dma_min_bytes > 0 ? ctx->cfg.dma_min_bytes : (8ll << 20);
+  const int64_t seg_bytes = pl.run_chunks * pl.C;
+  const bool bounce_ok = (int64_t)ln.half >= pl.C;
+  int variant = ctx->cfg.variant;
+  if (variant == TALARIA_VARIANT_AUTO) {
+    variant = TALARIA_VARIANT_ZEROCOPY;
+    if (bounce_ok && payload >= dma_min && seg_bytes >= (256 << 10)) variant = TALARIA_VARIANT_BOUNCE;
+    // a table of few long runs of adjacent ids needs no kernel at all
+    if (payload >= dma_min && (hl->stride_block == pl.C || n == 1)) {
+      const int64_t copies = pl.L * pl.P * count_id_runs(bt, n);
+      if (copies <= 1024 && payload / copies >= (1 << 20)) variant = TALARIA_VARIANT_RUNS;
+    }
+  }
+  if (variant == TALARIA_VARIANT_BOUNCE && !bounce_ok) variant = TALARIA_VARIANT_ZEROCOPY;
+  ctx->counters.last_variant = variant;
+
+  if (variant == TALARIA_VARIANT_ZEROCOPY) {
+    p.img = (char *)img_dev;
+    set_image_strides(p, pl.ord, hl->stride_layer, hl->stride_plane, hl->stride_block);
+    p.w0 = 0; p.w1 = pl.chunks;
+    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, zc_grid(ctx), stream));
+    return release_slot(ctx, slot, stream);
+  }
+
+  if (variant == TALARIA_VARIANT_RUNS) {
+    // one copy-engine copy per (layer, plane, run of adjacent ids); needs no descriptor
+    const bool blocks_contig = (hl->stride_block == pl.C) || n == 1;
+    for (int64_t l = 0; l < pl.L; ++l)
+      for (int64_t q = 0; q < pl.P; ++q) {
+        char *plane = (char *)kv->plane_base[l * pl.P + q];
+        int64_t i = 0;
+        while (i < n) {
+          int64_t j = i + 1;
+          if (blocks_contig)
+            while (j < n && bt[j] == bt[j - 1] + 1) ++j;
+          char *h = (char *)img + l * hl->stride_layer + q * hl->stride_plane + i * hl->stride_block;
+          char *d = plane + (int64_t)bt[i] * pl.C;
+          size_t bytes = (size_t)((j - i) * pl.C);
+          if (to_image) TAL_CUDA(ctx, cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, stream));
+          else          TAL_CUDA(ctx, cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, stream));
+          ctx->counters.memcpy_calls++;
+          i = j;
+        }
+      }
+    return release_slot(ctx, slot, stream);
+  }
+
+  // ---- bounce: kernel <-> device bounce half <-> large copy-engine copies ----
+  // The bounce half holds a piece of the image in image order, densely packed.
+  int64_t piece = (int64_t)ln.half / pl.C;                     // chunks per piece
+  if (pl.run_chunks < piece) piece = (piece / pl.run_chunks) * pl.run_chunks;
+  // dense image strides of the bounce copy: offset(w) = w*C
+  p.sd[0] = pl.C;
+  p.sd[1] = p.sd[0] * pl.ord.e0;
+  p.sd[2] = p.sd[1] * pl.ord.e1;
+
+  TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
+  for (int j = 0; j < 2; ++j) TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[j], ln.fork, 0));
+  int k = 0;
+  for (int64_t w0 = 0; w0 < pl.chunks; w0 += piece, ++k) {
+    const int64_t w1 = std::min(pl.chunks, w0 + piece);
+    const int j = k & 1;
+    char *half = ln.buf + (size_t)j * ln.half;
+    p.img = half - w0 * pl.C;   // so that offset(w) lands at (w - w0)*C inside the half
+    p.w0 = w0; p.w1 = w1;
+    if (to_image) TAL_TRY(launch_dir(ctx, true, p, pl.vec && ((uintptr_t)half % 16 == 0), hbm_grid(ctx, 512), ln.s[j]));
+    for (int64_t ws = w0; ws < w1;) {
+      int64_t we = std::min(w1, (ws / pl.run_chunks + 1) * pl.run_chunks);
+      char *h = (char *)img + image_offset(pl, hl, ws);
+      char *d = half + (ws - w0) * pl.C;
+      size_t bytes = (size_t)((we - ws) * pl.C);
+      if (to_image) TAL_CUDA(ctx, cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, ln.s[j]));
+      else          TAL_CUDA(ctx, cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, ln.s[j]));
+      ctx->counters.memcpy_calls++;
+      ws = we;
+    }
+    if (!to_image) TAL_TRY(launch_dir(ctx, false, p, pl.vec && ((uintptr_t)half % 16 == 0), hbm_grid(ctx, 512), ln.s[j]));
+  }
+  for (int j = 0; j < 2; ++j) {
+    TAL_CUDA(ctx, cudaEventRecord(ln.done[j], ln.s[j]));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[j], 0));
+  }
+  return release_slot(ctx, slot, stream);
+}
+
+}  // namespace tal
+
+using namespace tal;
+
+#define TAL_ENTER(ctx)                                   \
+  if (!(ctx)) return TALARIA_ERR_INVALID_ARG;            \
+  std::lock_guard<std::mutex> lk__((ctx)->mu);           \
+  DeviceGuard guard__((ctx)->device);                    \
+  if (!guard__.ok) return TALARIA_ERR_CUDA
+
+extern "C" talaria_status_t talaria_kv_offload(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                               const int32_t *block_table, int64_t first_block,
+                                               int64_t n_blocks, void *host_dst,
+                                               const talaria_host_layout_t *hl, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_transfer(ctx, kv, block_table, first_block, n_blocks, host_dst, hl, (cudaStream_t)stream, true, false);
+}
+
+extern "C" talaria_status_t talaria_kv_restore(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                               const int32_t *new_block_table, int64_t first_block,
+                                               int64_t n_blocks, const void *host_src,
+                                               const talaria_host_layout_t *hl, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_transfer(ctx, kv, new_block_table, first_block, n_blocks, (void *)host_src, hl,
+                     (cudaStream_t)stream, false, false);
+}
+
+extern "C" talaria_status_t talaria_kv_gather(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                              const int32_t *block_table, int64_t first_block,
+                                              int64_t n_blocks, void *d_image,
+                                              const talaria_host_layout_t *il, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_transfer(ctx, kv, block_table, first_block, n_blocks, d_image, il, (cudaStream_t)stream, true, true);
+}
+
+extern "C" talaria_status_t talaria_kv_scatter(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                               const int32_t *new_block_table, int64_t first_block,
+                                               int64_t n_blocks, const void *d_image,
+                                               const talaria_host_layout_t *il, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_transfer(ctx, kv, new_block_table, first_block, n_blocks, (void *)d_image, il,
+                     (cudaStream_t)stream, false, true);
+}
+
+// Restore tables of different sessions must not share a block either.
+static talaria_status_t batch_dup_check(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                        const talaria_kv_xfer_t *x, int32_t n) {
+  if (!ctx->cfg.validate || !kv || kv->num_blocks <= 0) return TALARIA_OK;
+  std::vector<uint64_t> bits((size_t)((kv->num_blocks + 63) / 64), 0);
+  for (int32_t s = 0; s < n; ++s) {
+    if (x[s].n_blocks < 0 || x[s].first_block < 0) return TALARIA_ERR_INVALID_ARG;
+    if (x[s].n_blocks == 0) continue;
+    if (!x[s].block_table) return TALARIA_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < x[s].n_blocks; ++i) {
+      int32_t b = x[s].block_table[x[s].first_block + i];
+      if (b < 0 || b >= kv->num_blocks) return TALARIA_ERR_BAD_BLOCK_ID;
+      uint64_t bit = 1ull << (b & 63);
+      if (bits[(size_t)b >> 6] & bit) return TALARIA_ERR_DUP_BLOCK;
+      bits[(size_t)b >> 6] |= bit;
+    }
+  }
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_kv_offload_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                                     const talaria_kv_xfer_t *xfers, int32_t n_xfers,
+                                                     void *stream) {
+  TAL_ENTER(ctx);
+  if (n_xfers < 0 || (n_xfers > 0 && !xfers)) return TALARIA_ERR_INVALID_ARG;
+  for (int32_t s = 0; s < n_xfers; ++s)
+    TAL_TRY(kv_transfer(ctx, kv, xfers[s].block_table, xfers[s].first_block, xfers[s].n_blocks,
+                        xfers[s].host, &xfers[s].hl, (cudaStream_t)stream, true, false));
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_kv_restore_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                                     const talaria_kv_xfer_t *xfers, int32_t n_xfers,
+                                                     void *stream) {
+  TAL_ENTER(ctx);
+  if (n_xfers < 0 || (n_xfers > 0 && !xfers)) return TALARIA_ERR_INVALID_ARG;
+  TAL_TRY(batch_dup_check(ctx, kv, xfers, n_xfers));
+  for (int32_t s = 0; s < n_xfers; ++s)
+    TAL_TRY(kv_transfer(ctx, kv, xfers[s].block_table, xfers[s].first_block, xfers[s].n_blocks,
+                        xfers[s].host, &xfers[s].hl, (cudaStream_t)stream, false, false));
+  return TALARIA_OK;
+}

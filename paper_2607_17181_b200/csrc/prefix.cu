@@ -1,0 +1,415 @@
+// Chained block hash and prefix match (Sec. 4.3 "cumulative prefix hash";
+// App. A "Prefix reuse"; App. B "at page boundaries").
+//
+//   digest_k = sum_j mix64(u32(tok[kB+j]) + G*(j+1));  s_k = s_{k-1}*P + digest_k;
+//   hash_k   = mix64(s_k)
+//
+// Two launches per call, whatever the number of pairs:
+//   1. tile kernel  -- a CTA per 2048-token tile of a pair: coalesced token loads,
+//      per-token mix, warp-shuffle segmented sum to one digest per block, and the
+//      first token position where the two streams differ inside the tile.
+//   2. chain kernel -- a CTA per pair: the affine recurrence s -> s*P + d is
+//      associative under composition, so it is evaluated as a block-wide scan
+//      (thread-serial runs, shuffle scan across lanes, shared memory across warps);
+//      then hash compare against the stored session's hashes, min-reductions for
+//      matched_blocks and the token LCP, and the result record.
+// No atomics, no inter-CTA waiting, bit-identical for any grid shape.
+#include <algorithm>
+#include <cstring>
+
+#include "internal.h"
+
+namespace tal {
+
+constexpr uint64_t kG = 0x9E3779B97F4A7C15ull;
+constexpr uint64_t kP = 0xD1342543DE82EF95ull;
+constexpr int kTileTok = 2048;
+constexpr int kTileThreads = 256;
+constexpr int kScanThreads = 256;
+constexpr int kScanItems = 8;
+constexpr long long kNoMismatch = 0x7fffffffffffffffll;
+
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+  z ^= z >> 30;
+  z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+struct PairDesc {
+  int64_t cont_off, sess_off;          // token offsets into the concatenated arrays
+  int64_t Tc, Ts;                      // token counts
+  int64_t cont_blk_off, sess_blk_off;  // block offsets into hash / digest arrays
+  int64_t tile_off;                    // first tile of this pair
+};
+
+struct PrefixParams {
+  const PairDesc *pairs;      // DEVICE [n_pairs + 1] (last entry holds the totals)
+  int32_t n_pairs;
+  int32_t B;
+  int32_t log2B;              // >= 0 when B is a power of two <= 32, else -1
+  int32_t need_sess_digest;   // 1 when stored hashes are not supplied
+  const int32_t *cont, *sess; // DEVICE tokens
+  uint64_t *dig_c, *dig_s;    // DEVICE scratch digests
+  long long *tile_mis;        // DEVICE scratch [total tiles]
+  const uint64_t *sess_hashes;// DEVICE or null
+  uint64_t *cont_hashes_out;  // DEVICE or null
+  talaria_match_t *results;   // DEVICE [n_pairs] or null
+  uint64_t seed;
+};
+
+__device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int m) {
+  return (uint64_t)__shfl_xor_sync(0xffffffffu, (unsigned long long)v, m);
+}
+__device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
+  return (uint64_t)__shfl_up_sync(0xffffffffu, (unsigned long long)v, d);
+}
+
+__global__ void __launch_bounds__(kTileThreads) prefix_tile_kernel(const __grid_constant__ PrefixParams p) {
+  __shared__ int s_pair;
+  __shared__ long long s_min[kTileThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) {
+    // last pair whose first tile is <= this tile
+    int lo = 0, hi = p.n_pairs - 1;
+    const long long t = blockIdx.x;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (p.pairs[mid].tile_off <= t) lo = mid; else hi = mid - 1;
+    }
+    s_pair = lo;
+  }
+  __syncthreads();
+  const PairDesc pd = p.pairs[s_pair];
+  const int64_t base = ((int64_t)blockIdx.x - pd.tile_off) * kTileTok;
+  const int32_t *cont = p.cont + pd.cont_off;
+  const int32_t *sess = p.sess + pd.sess_off;
+  const int64_t Tmin = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
+  const int B = p.B;
+  const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
+  long long first_mis = kNoMismatch;
+
+  if (p.log2B >= 0) {
+    // fast path: one token per thread per round; B consecutive lanes own one block
+#pragma unroll 4
+    for (int r = 0; r < kTileTok / kTileThreads; ++r) {
+      const int64_t g = base + r * kTileThreads + tid;
+      const int64_t k = g >> p.log2B;
+      const int j = (int)(g & (B - 1));
+      const uint64_t w = kG * (uint64_t)(j + 1);
+      int32_t tc = 0, ts = 0;
+      const bool hc = g < pd.Tc, hs = g < pd.Ts;
+      if (hc) tc = __ldg(cont + g);
+      if (hs) ts = __ldg(sess + g);
+      if (g < Tmin && tc != ts && first_mis == kNoMismatch) first_mis = g;
+      uint64_t vc = hc ? mix64((uint64_t)(uint32_t)tc + w) : 0ull;
+      uint64_t vs = (p.need_sess_digest && hs) ? mix64((uint64_t)(uint32_t)ts + w) : 0ull;
+      for (int m = 1; m < B; m <<= 1) {
+        vc += shfl_xor_u64(vc, m);
+        if (p.need_sess_digest) vs += shfl_xor_u64(vs, m);
+      }
+      if (j == 0) {
+        if (k < nbc) p.dig_c[pd.cont_blk_off + k] = vc;
+        if (p.need_sess_digest && k < nbs) p.dig_s[pd.sess_blk_off + k] = vs;
+      }
+    }
+  } else {
+    // general block size: a warp per block that STARTS inside this tile
+    for (int r = 0; r < kTileTok / kTileThreads; ++r) {
+      const int64_t g = base + r * kTileThreads + tid;
+      if (g < Tmin && first_mis == kNoMismatch && __ldg(cont + g) != __ldg(sess + g)) first_mis = g;
+    }
+    const int64_t k_first = (base + B - 1) / B;
+    const int64_t nb_max = nbc > nbs ? nbc : nbs;
+    for (int64_t k = k_first + wid; k < nb_max && k * B < base + kTileTok; k += kTileThreads / 32) {
+      const bool dc = k < nbc, ds = p.need_sess_digest && k < nbs;
+      uint64_t vc = 0, vs = 0;
+      for (int j = lane; j < B; j += 32) {
+        const uint64_t w = kG * (uint64_t)(j + 1);
+        if (dc) vc += mix64((uint64_t)(uint32_t)__ldg(cont + k * B + j) + w);
+        if (ds) vs += mix64((uint64_t)(uint32_t)__ldg(sess + k * B + j) + w);
+      }
+      for (int m = 16; m >= 1; m >>= 1) {
+        vc += shfl_xor_u64(vc, m);
+        vs += shfl_xor_u64(vs, m);
+      }
+      if (lane == 0) {
+        if (dc) p.dig_c[pd.cont_blk_off + k] = vc;
+        if (ds) p.dig_s[pd.sess_blk_off + k] = vs;
+      }
+    }
+  }
+
+  // first mismatch inside the tile
+  for (int m = 16; m >= 1; m >>= 1) {
+    long long o = __shfl_xor_sync(0xffffffffu, first_mis, m);
+    first_mis = o < first_mis ? o : first_mis;
+  }
+  if (lane == 0) s_min[wid] = first_mis;
+  __syncthreads();
+  if (tid == 0) {
+    long long v = s_min[0];
+    for (int k = 1; k < kTileThreads / 32; ++k) v = s_min[k] < v ? s_min[k] : v;
+    p.tile_mis[blockIdx.x] = v;
+  }
+}
+
+// (a1,b1) then (a2,b2):  x -> (x*a1 + b1)*a2 + b2
+struct Affine2 {
+  uint64_t a, bc, bs;
+};
+__device__ __forceinline__ Affine2 then(const Affine2 &f, const Affine2 &g) {
+  return Affine2{f.a * g.a, f.bc * g.a + g.bc, f.bs * g.a + g.bs};
+}
+
+__global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid_constant__ PrefixParams p) {
+  __shared__ Affine2 s_warp[kScanThreads / 32];
+  __shared__ uint64_t s_carry[2];
+  __shared__ long long s_red[kScanThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const PairDesc pd = p.pairs[blockIdx.x];
+  const int B = p.B;
+  const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
+  const int64_t lim = nbc < nbs ? nbc : nbs;                 // blocks that can be compared
+  const bool derive_s = p.need_sess_digest != 0;
+  const int64_t nb = derive_s ? (nbc > nbs ? nbc : nbs) : nbc;  // blocks to chain
+  const uint64_t *dc = p.dig_c + pd.cont_blk_off;
+  const uint64_t *ds = derive_s ? p.dig_s + pd.sess_blk_off : nullptr;
+  const uint64_t *hs_in = p.sess_hashes ? p.sess_hashes + pd.sess_blk_off : nullptr;
+  uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_blk_off : nullptr;
+
+  if (tid == 0) { s_carry[0] = p.seed; s_carry[1] = p.seed; }
+  __syncthreads();
+  long long first_bad = lim;
+
+  for (int64_t chunk = 0; chunk < nb; chunk += (int64_t)kScanThreads * kScanItems) {
+    const int64_t k0 = chunk + (int64_t)tid * kScanItems;
+    uint64_t vc[kScanItems], vs[kScanItems];
+    Affine2 loc{1ull, 0ull, 0ull};
+#pragma unroll
+    for (int q = 0; q < kScanItems; ++q) {
+      const int64_t k = k0 + q;
+      vc[q] = (k < nbc) ? dc[k] : 0ull;
+      vs[q] = (derive_s && k < nbs) ? ds[k] : 0ull;
+      if (k < nb) loc = Affine2{loc.a * kP, loc.bc * kP + vc[q], loc.bs * kP + vs[q]};
+    }
+    // inclusive scan across the warp
+    Affine2 inc = loc;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      Affine2 prev{shfl_up_u64(inc.a, d), shfl_up_u64(inc.bc, d), shfl_up_u64(inc.bs, d)};
+      if (lane >= d) inc = then(prev, inc);
+    }
+    if (lane == 31) s_warp[wid] = inc;
+    // exclusive prefix inside the warp
+    Affine2 exc{shfl_up_u64(inc.a, 1), shfl_up_u64(inc.bc, 1), shfl_up_u64(inc.bs, 1)};
+    if (lane == 0) exc = Affine2{1ull, 0ull, 0ull};
+    __syncthreads();
+    Affine2 before{1ull, 0ull, 0ull};
+    for (int w = 0; w < wid; ++w) before = then(before, s_warp[w]);
+    before = then(before, exc);
+    uint64_t sc = s_carry[0] * before.a + before.bc;
+    uint64_t ss = s_carry[1] * before.a + before.bs;
+#pragma unroll
+    for (int q = 0; q < kScanItems; ++q) {
+      const int64_t k = k0 + q;
+      if (k < nb) {
+        sc = sc * kP + vc[q];
+        ss = ss * kP + vs[q];
+        const uint64_t hc = mix64(sc);
+        if (k < nbc && hc_out) hc_out[k] = hc;
+        if (k < lim) {
+          const uint64_t hs = derive_s ? mix64(ss) : hs_in[k];
+          if (hs != hc && k < first_bad) first_bad = k;
+        }
+      }
+    }
+    __syncthreads();                       // everyone has read s_carry and s_warp
+    if (tid == kScanThreads - 1) { s_carry[0] = sc; s_carry[1] = ss; }
+    __syncthreads();
+  }
+
+  // token-level first mismatch over this pair's tiles
+  long long lcp = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
+  const int64_t t0 = pd.tile_off, t1 = p.pairs[blockIdx.x + 1].tile_off;
+  for (int64_t t = t0 + tid; t < t1; t += kScanThreads) {
+    long long v = p.tile_mis[t];
+    lcp = v < lcp ? v : lcp;
+  }
+  for (int m = 16; m >= 1; m >>= 1) {
+    long long o = __shfl_xor_sync(0xffffffffu, lcp, m);
+    lcp = o < lcp ? o : lcp;
+    long long o2 = __shfl_xor_sync(0xffffffffu, first_bad, m);
+    first_bad = o2 < first_bad ? o2 : first_bad;
+  }
+  __syncthreads();
+  if (lane == 0) s_red[wid] = lcp;
+  __syncthreads();
+  if (tid == 0) for (int w = 1; w < kScanThreads / 32; ++w) lcp = s_red[w] < lcp ? s_red[w] : lcp;
+  __syncthreads();
+  if (lane == 0) s_red[wid] = first_bad;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kScanThreads / 32; ++w) first_bad = s_red[w] < first_bad ? s_red[w] : first_bad;
+    if (p.results) {
+      const long long lcp_blocks = lcp / B;
+      const long long tok_blocks = lcp_blocks < lim ? lcp_blocks : lim;
+      talaria_match_t r;
+      r.lcp_tokens = lcp;
+      r.matched_blocks = first_bad;
+      r.reusable_tokens = (long long)B * (first_bad < lcp_blocks ? first_bad : lcp_blocks);
+      r.hash_token_disagree = (first_bad != tok_blocks) ? 1 : 0;
+      r.reserved = 0;
+      p.results[blockIdx.x] = r;
+    }
+  }
+}
+
+// Host side: validates offsets, builds the pair table, sizes scratch, launches.
+static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont,
+                                      const int64_t *cont_off, const int32_t *d_sess,
+                                      const int64_t *sess_off, const uint64_t *d_sess_hashes, int32_t B,
+                                      uint64_t seed, uint64_t *d_cont_hashes, talaria_match_t *d_results,
+                                      cudaStream_t stream) {
+  if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_pairs == 0) return TALARIA_OK;
+  if (!cont_off || !sess_off) return TALARIA_ERR_INVALID_ARG;
+  DescSlot *slot;
+  TAL_TRY(acquire_slot(ctx, (size_t)(n_pairs + 1) * sizeof(PairDesc), &slot));
+  PairDesc *pd = (PairDesc *)slot->h;
+  int64_t cb = 0, sb = 0, tiles = 0;
+  for (int32_t q = 0; q < n_pairs; ++q) {
+    int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
+    if (Tc < 0 || Ts < 0 || cont_off[q] < 0 || sess_off[q] < 0) return TALARIA_ERR_INVALID_ARG;
+    pd[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, tiles};
+    cb += Tc / B;
+    sb += Ts / B;
+    tiles += (std::max(Tc, Ts) + kTileTok - 1) / kTileTok;
+  }
+  pd[n_pairs] = PairDesc{cont_off[n_pairs], sess_off[n_pairs], 0, 0, cb, sb, tiles};
+  if (cont_off[n_pairs] > cont_off[0] && !d_cont) return TALARIA_ERR_INVALID_ARG;
+  if (sess_off[n_pairs] > sess_off[0] && !d_sess) return TALARIA_ERR_INVALID_ARG;
+  if (tiles > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
+
+  const bool derive = (d_sess_hashes == nullptr);
+  const size_t dig_c_bytes = (size_t)cb * 8, dig_s_bytes = derive ? (size_t)sb * 8 : 0;
+  const size_t need = dig_c_bytes + dig_s_bytes + (size_t)tiles * 8 + 64;
+  TAL_TRY(grow(ctx, &ctx->prefix_scratch, need));
+  TAL_TRY(upload_slot(ctx, slot, (size_t)(n_pairs + 1) * sizeof(PairDesc), stream));
+
+  PrefixParams p{};
+  p.pairs = (const PairDesc *)slot->d;
+  p.n_pairs = n_pairs;
+  p.B = B;
+  p.log2B = -1;
+  if (B <= 32 && (B & (B - 1)) == 0) {
+    int l = 0;
+    while ((1 << l) < B) ++l;
+    p.log2B = l;
+  }
+  p.need_sess_digest = derive ? 1 : 0;
+  p.cont = d_cont;
+  p.sess = d_sess;
+  p.dig_c = (uint64_t *)ctx->prefix_scratch.p;
+  p.dig_s = (uint64_t *)(ctx->prefix_scratch.p + dig_c_bytes);
+  p.tile_mis = (long long *)(ctx->prefix_scratch.p + dig_c_bytes + dig_s_bytes);
+  p.sess_hashes = d_sess_hashes;
+  p.cont_hashes_out = d_cont_hashes;
+  p.results = d_results;
+  p.seed = seed;
+  if (tiles > 0) {
+    prefix_tile_kernel<<<(unsigned)tiles, kTileThreads, 0, stream>>>(p);
+    TAL_CUDA(ctx, cudaGetLastError());
+    ctx->counters.kernel_launches++;
+  }
+  prefix_chain_kernel<<<(unsigned)n_pairs, kScanThreads, 0, stream>>>(p);
+  TAL_CUDA(ctx, cudaGetLastError());
+  ctx->counters.kernel_launches++;
+  return release_slot(ctx, slot, stream);
+}
+
+}  // namespace tal
+
+using namespace tal;
+
+#define TAL_ENTER(ctx)                                   \
+  if (!(ctx)) return TALARIA_ERR_INVALID_ARG;            \
+  std::lock_guard<std::mutex> lk__((ctx)->mu);           \
+  DeviceGuard guard__((ctx)->device);                    \
+  if (!guard__.ok) return TALARIA_ERR_CUDA
+
+extern "C" talaria_status_t talaria_block_hash(talaria_ctx *ctx, const int32_t *d_tokens, int64_t n_tokens,
+                                               int32_t block_tokens, uint64_t seed,
+                                               uint64_t *d_hashes_out, void *stream) {
+  TAL_ENTER(ctx);
+  if (n_tokens < 0 || block_tokens <= 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_tokens / block_tokens == 0) return TALARIA_OK;
+  if (!d_tokens || !d_hashes_out) return TALARIA_ERR_INVALID_ARG;
+  const int64_t co[2] = {0, n_tokens}, so[2] = {0, 0};
+  return prefix_launch(ctx, 1, d_tokens, co, d_tokens, so, nullptr, block_tokens, seed, d_hashes_out,
+                       nullptr, (cudaStream_t)stream);
+}
+
+extern "C" talaria_status_t talaria_prefix_match(talaria_ctx *ctx, int32_t n_pairs,
+                                                 const int32_t *d_cont_tokens, const int64_t *cont_offsets,
+                                                 const int32_t *d_sess_tokens, const int64_t *sess_offsets,
+                                                 const uint64_t *d_sess_hashes, int32_t block_tokens,
+                                                 uint64_t seed, uint64_t *d_cont_hashes_out,
+                                                 talaria_match_t *d_results, void *stream) {
+  TAL_ENTER(ctx);
+  if (n_pairs > 0 && !d_results) return TALARIA_ERR_INVALID_ARG;
+  return prefix_launch(ctx, n_pairs, d_cont_tokens, cont_offsets, d_sess_tokens, sess_offsets,
+                       d_sess_hashes, block_tokens, seed, d_cont_hashes_out, d_results,
+                       (cudaStream_t)stream);
+}
+
+extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
+                                                      const int32_t *h_cont, const int64_t *cont_offsets,
+                                                      const int32_t *h_sess, const int64_t *sess_offsets,
+                                                      const uint64_t *h_sess_hashes, int32_t B,
+                                                      uint64_t seed, uint64_t *h_cont_hashes_out,
+                                                      talaria_match_t *h_results, void *stream_) {
+  TAL_ENTER(ctx);
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_pairs == 0) return TALARIA_OK;
+  if (!cont_offsets || !sess_offsets || !h_results) return TALARIA_ERR_INVALID_ARG;
+  const int64_t c0 = cont_offsets[0], s0 = sess_offsets[0];
+  const int64_t nc = cont_offsets[n_pairs] - c0, ns = sess_offsets[n_pairs] - s0;
+  if (nc < 0 || ns < 0 || (nc > 0 && !h_cont) || (ns > 0 && !h_sess)) return TALARIA_ERR_INVALID_ARG;
+  int64_t cb = 0, sb = 0;
+  std::vector<int64_t> co(n_pairs + 1), so(n_pairs + 1);
+  for (int32_t q = 0; q <= n_pairs; ++q) {
+    co[q] = cont_offsets[q] - c0;
+    so[q] = sess_offsets[q] - s0;
+    if (q < n_pairs) {
+      int64_t Tc = cont_offsets[q + 1] - cont_offsets[q], Ts = sess_offsets[q + 1] - sess_offsets[q];
+      if (Tc < 0 || Ts < 0) return TALARIA_ERR_INVALID_ARG;
+      cb += Tc / B;
+      sb += Ts / B;
+    }
+  }
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  const size_t o_cont = 0, o_sess = o_cont + up((size_t)nc * 4), o_sh = o_sess + up((size_t)ns * 4),
+               o_ch = o_sh + up(h_sess_hashes ? (size_t)sb * 8 : 0), o_res = o_ch + up((size_t)cb * 8),
+               total = o_res + up((size_t)n_pairs * sizeof(talaria_match_t));
+  TAL_TRY(grow(ctx, &ctx->host_tok, total));
+  char *d = ctx->host_tok.p;
+  if (nc) TAL_CUDA(ctx, cudaMemcpyAsync(d + o_cont, h_cont + c0, (size_t)nc * 4, cudaMemcpyHostToDevice, stream));
+  if (ns) TAL_CUDA(ctx, cudaMemcpyAsync(d + o_sess, h_sess + s0, (size_t)ns * 4, cudaMemcpyHostToDevice, stream));
+  if (h_sess_hashes && sb)
+    TAL_CUDA(ctx, cudaMemcpyAsync(d + o_sh, h_sess_hashes, (size_t)sb * 8, cudaMemcpyHostToDevice, stream));
+  ctx->counters.memcpy_calls += 3;
+  TAL_TRY(prefix_launch(ctx, n_pairs, (const int32_t *)(d + o_cont), co.data(), (const int32_t *)(d + o_sess),
+                        so.data(), h_sess_hashes ? (const uint64_t *)(d + o_sh) : nullptr, B, seed,
+                        (uint64_t *)(d + o_ch), (talaria_match_t *)(d + o_res), stream));
+  if (h_cont_hashes_out && cb)
+    TAL_CUDA(ctx, cudaMemcpyAsync(h_cont_hashes_out, d + o_ch, (size_t)cb * 8, cudaMemcpyDeviceToHost, stream));
+  TAL_CUDA(ctx, cudaMemcpyAsync(h_results, d + o_res, (size_t)n_pairs * sizeof(talaria_match_t),
+                                cudaMemcpyDeviceToHost, stream));
+  ctx->counters.memcpy_calls += 2;
+  TAL_CUDA(ctx, cudaStreamSynchronize(stream));
+  return TALARIA_OK;
+}

@@ -1,0 +1,215 @@
+// Staged switching (Sec. 4.4): clean staged chunks move device-to-device into
+// their stable-address slots, dirty or missing chunks are reloaded from the
+// pinned host copy (App. D: "reloads those chunks from host rather than copying
+// unsafe D2D sources").
+//
+// The D2D leg is one persistent kernel over the whole plan: the plan is cut into
+// 32 KiB tiles, every CTA takes one contiguous span of tiles (so it streams
+// through memory and needs a single binary search to find its first entry), and
+// moves each tile with four 16-byte loads per thread in flight.  The H2D leg is
+// issued on an internal stream as copy-engine copies, merged over neighbouring
+// chunks, and overlaps the kernel.
+#include <algorithm>
+#include <cstring>
+
+#include "internal.h"
+
+namespace tal {
+
+struct StageEntry {
+  const char *src;
+  char *dst;
+  int64_t bytes;
+  int64_t tile0;    // first tile of this entry
+};
+
+constexpr int kStageThreads = 512;
+constexpr int kStageTile = kStageThreads * 16 * 4;   // 32 KiB
+
+struct StageParams {
+  const StageEntry *entries;   // DEVICE [n + 1]; entries[n].tile0 = total tiles
+  int64_t n;
+  int64_t tiles;
+};
+
+__global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_constant__ StageParams p) {
+  __shared__ int64_t s_entry;
+  const int tid = threadIdx.x;
+  // contiguous span of tiles for this CTA
+  const int64_t per = p.tiles / gridDim.x, rem = p.tiles % gridDim.x;
+  const int64_t b = blockIdx.x;
+  const int64_t t_begin = b * per + (b < rem ? b : rem);
+  const int64_t t_end = t_begin + per + (b < rem ? 1 : 0);
+  if (t_begin >= t_end) return;
+  if (tid == 0) {
+    int64_t lo = 0, hi = p.n - 1;       // last entry with tile0 <= t_begin
+    while (lo < hi) {
+      int64_t mid = (lo + hi + 1) >> 1;
+      if (p.entries[mid].tile0 <= t_begin) lo = mid; else hi = mid - 1;
+    }
+    s_entry = lo;
+  }
+  __syncthreads();
+  int64_t e = s_entry;
+  StageEntry cur = p.entries[e];
+  int64_t next_tile0 = p.entries[e + 1].tile0;
+  for (int64_t t = t_begin; t < t_end; ++t) {
+    while (t >= next_tile0) {            // entries with zero tiles are skipped too
+      ++e;
+      cur = p.entries[e];
+      next_tile0 = p.entries[e + 1].tile0;
+    }
+    const int64_t off = (t - cur.tile0) * kStageTile;
+    const int64_t len = min((int64_t)kStageTile, cur.bytes - off);
+    const char *src = cur.src + off;
+    char *dst = cur.dst + off;
+    if ((((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
+      const int4 *s4 = (const int4 *)src;
+      int4 *d4 = (int4 *)dst;
+      if (len == kStageTile) {
+        int4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) v[k] = __ldcs(s4 + tid + k * kStageThreads);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) __stcs(d4 + tid + k * kStageThreads, v[k]);
+      } else {
+        const int n16 = (int)(len >> 4);
+        for (int k = tid; k < n16; k += kStageThreads) __stcs(d4 + k, __ldcs(s4 + k));
+        for (int k = (n16 << 4) + tid; k < len; k += kStageThreads) dst[k] = src[k];
+      }
+    } else {
+      for (int k = tid; k < len; k += kStageThreads) dst[k] = src[k];
+    }
+  }
+}
+
+struct Range {
+  uintptr_t lo, hi;
+};
+
+static bool any_overlap_sorted(std::vector<Range> &a) {
+  std::sort(a.begin(), a.end(), [](const Range &x, const Range &y) { return x.lo < y.lo; });
+  for (size_t k = 1; k < a.size(); ++k)
+    if (a[k].lo < a[k - 1].hi) return true;
+  return false;
+}
+
+// a sorted & disjoint; does any range of b intersect a range of a?
+static bool cross_overlap(const std::vector<Range> &a, std::vector<Range> &b) {
+  std::sort(b.begin(), b.end(), [](const Range &x, const Range &y) { return x.lo < y.lo; });
+  size_t i = 0;
+  for (const Range &r : b) {
+    while (i < a.size() && a[i].hi <= r.lo) ++i;
+    // b is sorted by lo but its ranges may overlap each other, so look back as well
+    size_t j = i;
+    if (j < a.size() && a[j].lo < r.hi && r.lo < a[j].hi) return true;
+  }
+  return false;
+}
+
+static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                   const uint8_t *dirty, talaria_stage_stats_t *stats, cudaStream_t stream) {
+  if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
+  talaria_stage_stats_t st{0, 0, 0, 0};
+  if (n == 0) {
+    if (stats) *stats = st;
+    return TALARIA_OK;
+  }
+  // classify
+  std::vector<uint8_t> from_host((size_t)n, 0);
+  int64_t n_clean = 0;
+  for (int64_t k = 0; k < n; ++k) {
+    const talaria_copy_t &c = plan[k];
+    if (c.bytes < 0 || !c.dst_dev) return TALARIA_ERR_INVALID_ARG;
+    const bool missing = (c.src_dev == nullptr);
+    const bool is_dirty = !missing && dirty && c.chunk_id >= 0 && ((dirty[c.chunk_id >> 3] >> (c.chunk_id & 7)) & 1);
+    if (missing || is_dirty) {
+      if (!c.src_host) return TALARIA_ERR_INVALID_ARG;
+      from_host[(size_t)k] = 1;
+      st.h2d_bytes += c.bytes;
+      if (missing) st.missing_chunks++; else st.dirty_chunks++;
+    } else {
+      st.d2d_bytes += c.bytes;
+      ++n_clean;
+    }
+  }
+  if (ctx->cfg.validate) {
+    std::vector<Range> dsts, srcs;
+    dsts.reserve((size_t)n);
+    srcs.reserve((size_t)n_clean);
+    for (int64_t k = 0; k < n; ++k) {
+      if (plan[k].bytes == 0) continue;
+      dsts.push_back({(uintptr_t)plan[k].dst_dev, (uintptr_t)plan[k].dst_dev + (uintptr_t)plan[k].bytes});
+      if (!from_host[(size_t)k])
+        srcs.push_back({(uintptr_t)plan[k].src_dev, (uintptr_t)plan[k].src_dev + (uintptr_t)plan[k].bytes});
+    }
+    if (any_overlap_sorted(dsts)) return TALARIA_ERR_OVERLAP;
+    if (cross_overlap(dsts, srcs)) return TALARIA_ERR_OVERLAP;
+  }
+
+  // ---- H2D leg: merged copy-engine copies on an internal stream ----------
+  BounceLane &ln = ctx->lane[1];
+  bool forked = false;
+  for (int64_t k = 0; k < n;) {
+    if (!from_host[(size_t)k] || plan[k].bytes == 0) { ++k; continue; }
+    const char *h = (const char *)plan[k].src_host;
+    char *d = (char *)plan[k].dst_dev;
+    int64_t bytes = plan[k].bytes;
+    int64_t j = k + 1;
+    while (j < n && from_host[(size_t)j] && (const char *)plan[j].src_host == h + bytes &&
+           (char *)plan[j].dst_dev == d + bytes) {
+      bytes += plan[j].bytes;
+      ++j;
+    }
+    void *alias;
+    TAL_TRY(mapped_pointer(ctx, h, &alias));
+    if (!forked) {
+      TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
+      TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
+      forked = true;
+    }
+    TAL_CUDA(ctx, cudaMemcpyAsync(d, h, (size_t)bytes, cudaMemcpyHostToDevice, ln.s[0]));
+    ctx->counters.memcpy_calls++;
+    k = j;
+  }
+
+  // ---- D2D leg ---------------------------------------------------------------
+  if (n_clean > 0 && st.d2d_bytes > 0) {
+    DescSlot *slot;
+    TAL_TRY(acquire_slot(ctx, (size_t)(n_clean + 1) * sizeof(StageEntry), &slot));
+    StageEntry *e = (StageEntry *)slot->h;
+    int64_t m = 0, tiles = 0;
+    for (int64_t k = 0; k < n; ++k) {
+      if (from_host[(size_t)k]) continue;
+      e[m++] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, tiles};
+      tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
+    }
+    e[m] = StageEntry{nullptr, nullptr, 0, tiles};
+    TAL_TRY(upload_slot(ctx, slot, (size_t)(m + 1) * sizeof(StageEntry), stream));
+    StageParams p{(const StageEntry *)slot->d, m, tiles};
+    int grid = (int)std::min<int64_t>(tiles, hbm_grid(ctx, kStageThreads));
+    stage_copy_kernel<<<grid, kStageThreads, 0, stream>>>(p);
+    TAL_CUDA(ctx, cudaGetLastError());
+    ctx->counters.kernel_launches++;
+    TAL_TRY(release_slot(ctx, slot, stream));
+  }
+  if (forked) {
+    TAL_CUDA(ctx, cudaEventRecord(ln.done[0], ln.s[0]));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[0], 0));
+  }
+  ctx->counters.payload_bytes += st.d2d_bytes + st.h2d_bytes;
+  if (stats) *stats = st;
+  return TALARIA_OK;
+}
+
+}  // namespace tal
+
+extern "C" talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                          const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
+                                          void *stream) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  tal::DeviceGuard g(ctx->device);
+  if (!g.ok) return TALARIA_ERR_CUDA;
+  return tal::stage_impl(ctx, plan, n, dirty_bitmap, stats, (cudaStream_t)stream);
+}
