@@ -158,9 +158,14 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
     TAL_CUDA(ctx, cudaGetDeviceProperties(&prop, device));
     ctx->sm_count = prop.multiProcessorCount;
     for (auto &s : ctx->ring) TAL_CUDA(ctx, cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming));
+    // Internal streams run at the highest priority: their kernels are short packing
+    // steps that gate copy-engine transfers, so they should not queue behind a long
+    // kernel of the caller's (for example a staging copy on another stream).
+    int prio_least = 0, prio_greatest = 0;
+    TAL_CUDA(ctx, cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
     for (auto &ln : ctx->lane) {
       for (int j = 0; j < 2; ++j) {
-        TAL_CUDA(ctx, cudaStreamCreateWithFlags(&ln.s[j], cudaStreamNonBlocking));
+        TAL_CUDA(ctx, cudaStreamCreateWithPriority(&ln.s[j], cudaStreamNonBlocking, prio_greatest));
         TAL_CUDA(ctx, cudaEventCreateWithFlags(&ln.done[j], cudaEventDisableTiming));
       }
       TAL_CUDA(ctx, cudaEventCreateWithFlags(&ln.fork, cudaEventDisableTiming));

@@ -3,12 +3,15 @@
 // pinned host copy (App. D: "reloads those chunks from host rather than copying
 // unsafe D2D sources").
 //
-// The D2D leg is one persistent kernel over the whole plan: the plan is cut into
-// 32 KiB tiles, every CTA takes one contiguous span of tiles (so it streams
-// through memory and needs a single binary search to find its first entry), and
-// moves each tile with four 16-byte loads per thread in flight.  The H2D leg is
-// issued on an internal stream as copy-engine copies, merged over neighbouring
-// chunks, and overlaps the kernel.
+// The D2D leg is one kernel over the whole plan: the plan is cut into 32 KiB tiles
+// and every CTA takes one short contiguous span of tiles (512 KiB), moving each
+// tile with four 16-byte loads per thread in flight.  The grid is NOT persistent
+// on purpose: staging runs next to KV offload / restore on other streams, and
+// short CTAs let the hardware scheduler interleave those kernels instead of
+// making them wait for a resident grid to drain.  The host precomputes the plan
+// entry each span starts in, so no CTA searches.  The H2D leg is issued on an
+// internal stream as copy-engine copies, merged over neighbouring chunks, and
+// overlaps the kernel.
 #include <algorithm>
 #include <cstring>
 
@@ -25,32 +28,20 @@ struct StageEntry {
 
 constexpr int kStageThreads = 512;
 constexpr int kStageTile = kStageThreads * 16 * 4;   // 32 KiB
+constexpr int kSpanTiles = 16;                       // tiles per CTA (512 KiB)
 
 struct StageParams {
   const StageEntry *entries;   // DEVICE [n + 1]; entries[n].tile0 = total tiles
+  const int32_t *span_entry;   // DEVICE [grid]: entry that holds the span's first tile
   int64_t n;
   int64_t tiles;
 };
 
 __global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_constant__ StageParams p) {
-  __shared__ int64_t s_entry;
   const int tid = threadIdx.x;
-  // contiguous span of tiles for this CTA
-  const int64_t per = p.tiles / gridDim.x, rem = p.tiles % gridDim.x;
-  const int64_t b = blockIdx.x;
-  const int64_t t_begin = b * per + (b < rem ? b : rem);
-  const int64_t t_end = t_begin + per + (b < rem ? 1 : 0);
-  if (t_begin >= t_end) return;
-  if (tid == 0) {
-    int64_t lo = 0, hi = p.n - 1;       // last entry with tile0 <= t_begin
-    while (lo < hi) {
-      int64_t mid = (lo + hi + 1) >> 1;
-      if (p.entries[mid].tile0 <= t_begin) lo = mid; else hi = mid - 1;
-    }
-    s_entry = lo;
-  }
-  __syncthreads();
-  int64_t e = s_entry;
+  const int64_t t_begin = (int64_t)blockIdx.x * kSpanTiles;
+  const int64_t t_end = min(p.tiles, t_begin + kSpanTiles);
+  int64_t e = p.span_entry[blockIdx.x];
   StageEntry cur = p.entries[e];
   int64_t next_tile0 = p.entries[e + 1].tile0;
   for (int64_t t = t_begin; t < t_end; ++t) {
@@ -148,47 +139,63 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   }
 
   // ---- H2D leg: merged copy-engine copies on an internal stream ----------
-  BounceLane &ln = ctx->lane[1];
-  bool forked = false;
+  // Every host source is checked before anything is enqueued, so a rejected plan
+  // leaves no partial copy behind.
+  struct HostRun { const char *h; char *d; int64_t bytes; };
+  std::vector<HostRun> runs;
   for (int64_t k = 0; k < n;) {
     if (!from_host[(size_t)k] || plan[k].bytes == 0) { ++k; continue; }
-    const char *h = (const char *)plan[k].src_host;
-    char *d = (char *)plan[k].dst_dev;
-    int64_t bytes = plan[k].bytes;
+    HostRun r{(const char *)plan[k].src_host, (char *)plan[k].dst_dev, plan[k].bytes};
     int64_t j = k + 1;
-    while (j < n && from_host[(size_t)j] && (const char *)plan[j].src_host == h + bytes &&
-           (char *)plan[j].dst_dev == d + bytes) {
-      bytes += plan[j].bytes;
+    while (j < n && from_host[(size_t)j] && (const char *)plan[j].src_host == r.h + r.bytes &&
+           (char *)plan[j].dst_dev == r.d + r.bytes) {
+      r.bytes += plan[j].bytes;
       ++j;
     }
     void *alias;
-    TAL_TRY(mapped_pointer(ctx, h, &alias));
-    if (!forked) {
-      TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
-      TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
-      forked = true;
-    }
-    TAL_CUDA(ctx, cudaMemcpyAsync(d, h, (size_t)bytes, cudaMemcpyHostToDevice, ln.s[0]));
-    ctx->counters.memcpy_calls++;
+    TAL_TRY(mapped_pointer(ctx, r.h, &alias));
+    runs.push_back(r);
     k = j;
+  }
+  BounceLane &ln = ctx->lane[1];
+  const bool forked = !runs.empty();
+  if (forked) {
+    TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
+    for (const HostRun &r : runs) {
+      TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
+      ctx->counters.memcpy_calls++;
+    }
   }
 
   // ---- D2D leg ---------------------------------------------------------------
   if (n_clean > 0 && st.d2d_bytes > 0) {
+    // count tiles first so the descriptor (entries, then one int32 per span) can be sized
+    int64_t tiles = 0;
+    for (int64_t k = 0; k < n; ++k)
+      if (!from_host[(size_t)k]) tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
+    const int64_t spans = (tiles + kSpanTiles - 1) / kSpanTiles;
+    if (spans > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
+    const size_t ent_bytes = ((size_t)(n_clean + 1) * sizeof(StageEntry) + 15) & ~(size_t)15;
+    const size_t desc_bytes = ent_bytes + (size_t)spans * sizeof(int32_t);
     DescSlot *slot;
-    TAL_TRY(acquire_slot(ctx, (size_t)(n_clean + 1) * sizeof(StageEntry), &slot));
+    TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
     StageEntry *e = (StageEntry *)slot->h;
-    int64_t m = 0, tiles = 0;
+    int32_t *span_entry = (int32_t *)(slot->h + ent_bytes);
+    int64_t m = 0, t0 = 0, next_span = 0;
     for (int64_t k = 0; k < n; ++k) {
       if (from_host[(size_t)k]) continue;
-      e[m++] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, tiles};
-      tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
+      const int64_t nt = (plan[k].bytes + kStageTile - 1) / kStageTile;
+      e[m] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, t0};
+      // spans whose first tile falls inside this entry
+      while (next_span < spans && next_span * kSpanTiles < t0 + nt) span_entry[next_span++] = (int32_t)m;
+      t0 += nt;
+      ++m;
     }
     e[m] = StageEntry{nullptr, nullptr, 0, tiles};
-    TAL_TRY(upload_slot(ctx, slot, (size_t)(m + 1) * sizeof(StageEntry), stream));
-    StageParams p{(const StageEntry *)slot->d, m, tiles};
-    int grid = (int)std::min<int64_t>(tiles, hbm_grid(ctx, kStageThreads));
-    stage_copy_kernel<<<grid, kStageThreads, 0, stream>>>(p);
+    TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+    StageParams p{(const StageEntry *)slot->d, (const int32_t *)(slot->d + ent_bytes), m, tiles};
+    stage_copy_kernel<<<(unsigned)spans, kStageThreads, 0, stream>>>(p);
     TAL_CUDA(ctx, cudaGetLastError());
     ctx->counters.kernel_launches++;
     TAL_TRY(release_slot(ctx, slot, stream));
