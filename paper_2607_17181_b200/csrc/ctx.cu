@@ -22,14 +22,24 @@ talaria_status_t acquire_slot(talaria_ctx *ctx, size_t bytes, DescSlot **out) {
     s.used = false;
   }
   if (s.cap < bytes) {
-    size_t cap = std::max<size_t>(bytes + bytes / 2, 64 << 10);
-    if (s.h) cudaFreeHost(s.h);
-    if (s.d) cudaFree(s.d);
-    s.h = s.d = nullptr;
-    s.cap = 0;
-    TAL_CUDA(ctx, cudaHostAlloc((void **)&s.h, cap, cudaHostAllocDefault));
-    TAL_CUDA(ctx, cudaMalloc((void **)&s.d, cap));
-    s.cap = cap;
+    // Growing frees device memory, which makes the whole device wait.  Do it once for
+    // the whole ring so the stall cannot recur slot by slot while other streams
+    // are busy.
+    const size_t cap = std::max<size_t>(bytes + bytes / 2, kSlotBytes);
+    for (DescSlot &r : ctx->ring) {
+      if (r.cap >= cap) continue;
+      if (r.used) {
+        TAL_CUDA(ctx, cudaEventSynchronize(r.ev));
+        r.used = false;
+      }
+      if (r.h) cudaFreeHost(r.h);
+      if (r.d) cudaFree(r.d);
+      r.h = r.d = nullptr;
+      r.cap = 0;
+      TAL_CUDA(ctx, cudaHostAlloc((void **)&r.h, cap, cudaHostAllocDefault));
+      TAL_CUDA(ctx, cudaMalloc((void **)&r.d, cap));
+      r.cap = cap;
+    }
   }
   *out = &s;
   return TALARIA_OK;
@@ -157,7 +167,12 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
     cudaDeviceProp prop{};
     TAL_CUDA(ctx, cudaGetDeviceProperties(&prop, device));
     ctx->sm_count = prop.multiProcessorCount;
-    for (auto &s : ctx->ring) TAL_CUDA(ctx, cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming));
+    for (auto &s : ctx->ring) {
+      TAL_CUDA(ctx, cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming));
+      TAL_CUDA(ctx, cudaHostAlloc((void **)&s.h, kSlotBytes, cudaHostAllocDefault));
+      TAL_CUDA(ctx, cudaMalloc((void **)&s.d, kSlotBytes));
+      s.cap = kSlotBytes;
+    }
     // Internal streams run at the highest priority: their kernels are short packing
     // steps that gate copy-engine transfers, so they should not queue behind a long
     // kernel of the caller's (for example a staging copy on another stream).

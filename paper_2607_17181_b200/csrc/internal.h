@@ -11,6 +11,7 @@
 namespace tal {
 
 constexpr int kRing = 8;              // descriptor slots in flight
+constexpr size_t kSlotBytes = 2u << 20;  // initial size of each slot (pinned + device)
 constexpr int kLanes = 2;             // 0: offload (device->host), 1: restore (host->device)
 
 struct DescSlot {

@@ -5,9 +5,10 @@
 //   hash_k   = mix64(s_k)
 //
 // Two launches per call, whatever the number of pairs:
-//   1. tile kernel  -- a CTA per 2048-token tile of a pair: coalesced token loads,
-//      per-token mix, warp-shuffle segmented sum to one digest per block, and the
-//      first token position where the two streams differ inside the tile.
+//   1. tile kernel  -- a CTA per 2048-token tile of a pair: coalesced 16-byte token
+//      loads (four tokens per thread, summed in registers), a warp-shuffle
+//      segmented sum over the B/4 lanes that share a block, and the first token
+//      position where the two streams differ inside the tile.
 //   2. chain kernel -- a CTA per pair: the affine recurrence s -> s*P + d is
 //      associative under composition, so it is evaluated as a block-wide scan
 //      (thread-serial runs, shuffle scan across lanes, shared memory across warps);
@@ -45,8 +46,12 @@ struct PairDesc {
   int64_t tile_off;                    // first tile of this pair
 };
 
+constexpr int kInlinePairs = 8;    // up to this many pairs travel in the kernel parameters
+
 struct PrefixParams {
-  const PairDesc *pairs;      // DEVICE [n_pairs + 1] (last entry holds the totals)
+  const PairDesc *pairs;      // DEVICE [n_pairs + 1] (last entry holds the totals); null when inline
+  const int32_t *tile_pair;   // DEVICE [tiles]: pair of each tile; null when inline
+  PairDesc inl[kInlinePairs + 1];
   int32_t n_pairs;
   int32_t B;
   int32_t log2B;              // >= 0 when B is a power of two <= 32, else -1
@@ -68,21 +73,17 @@ __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
 }
 
 __global__ void __launch_bounds__(kTileThreads) prefix_tile_kernel(const __grid_constant__ PrefixParams p) {
-  __shared__ int s_pair;
   __shared__ long long s_min[kTileThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  if (tid == 0) {
-    // last pair whose first tile is <= this tile
-    int lo = 0, hi = p.n_pairs - 1;
-    const long long t = blockIdx.x;
-    while (lo < hi) {
-      int mid = (lo + hi + 1) >> 1;
-      if (p.pairs[mid].tile_off <= t) lo = mid; else hi = mid - 1;
-    }
-    s_pair = lo;
+  int q = 0;
+  if (p.pairs) {
+    q = p.tile_pair[blockIdx.x];
+  } else {
+    // last inline pair whose first tile is <= this tile
+    for (int k = 1; k < p.n_pairs; ++k)
+      if (p.inl[k].tile_off <= (int64_t)blockIdx.x) q = k;
   }
-  __syncthreads();
-  const PairDesc pd = p.pairs[s_pair];
+  const PairDesc pd = p.pairs ? p.pairs[q] : p.inl[q];
   const int64_t base = ((int64_t)blockIdx.x - pd.tile_off) * kTileTok;
   const int32_t *cont = p.cont + pd.cont_off;
   const int32_t *sess = p.sess + pd.sess_off;
@@ -91,8 +92,53 @@ __global__ void __launch_bounds__(kTileThreads) prefix_tile_kernel(const __grid_
   const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
   long long first_mis = kNoMismatch;
 
-  if (p.log2B >= 0) {
-    // fast path: one token per thread per round; B consecutive lanes own one block
+  const bool vec_ok = p.log2B >= 2 && ((((uintptr_t)cont) | ((uintptr_t)sess)) & 15) == 0;
+  if (vec_ok) {
+    // four consecutive tokens per thread (one 16-byte load per stream); the B/4 lanes
+    // that share a block finish the sum with xor-shuffles
+    const int lanes_per_block = B >> 2;
+#pragma unroll
+    for (int r = 0; r < kTileTok / (kTileThreads * 4); ++r) {
+      const int64_t g0 = base + ((int64_t)r * kTileThreads + tid) * 4;
+      const int64_t k = g0 >> p.log2B;
+      const int j0 = (int)(g0 & (B - 1));
+      int tc[4] = {0, 0, 0, 0}, ts[4] = {0, 0, 0, 0};
+      if (g0 + 4 <= pd.Tc) {
+        const int4 v = __ldg((const int4 *)(cont + g0));
+        tc[0] = v.x; tc[1] = v.y; tc[2] = v.z; tc[3] = v.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) if (g0 + e < pd.Tc) tc[e] = __ldg(cont + g0 + e);
+      }
+      if (g0 + 4 <= pd.Ts) {
+        const int4 v = __ldg((const int4 *)(sess + g0));
+        ts[0] = v.x; ts[1] = v.y; ts[2] = v.z; ts[3] = v.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) if (g0 + e < pd.Ts) ts[e] = __ldg(sess + g0 + e);
+      }
+      uint64_t vc = 0, vs = 0;
+#pragma unroll
+      for (int e = 3; e >= 0; --e)
+        if (g0 + e < Tmin && tc[e] != ts[e]) first_mis = (first_mis < g0 + e) ? first_mis : g0 + e;
+      const bool full_c = k < nbc, full_s = p.need_sess_digest && k < nbs;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint64_t w = kG * (uint64_t)(j0 + e + 1);
+        if (full_c) vc += mix64((uint64_t)(uint32_t)tc[e] + w);
+        if (full_s) vs += mix64((uint64_t)(uint32_t)ts[e] + w);
+      }
+      for (int m = 1; m < lanes_per_block; m <<= 1) {
+        vc += shfl_xor_u64(vc, m);
+        if (p.need_sess_digest) vs += shfl_xor_u64(vs, m);
+      }
+      if (j0 == 0) {
+        if (full_c) p.dig_c[pd.cont_blk_off + k] = vc;
+        if (full_s) p.dig_s[pd.sess_blk_off + k] = vs;
+      }
+    }
+  } else if (p.log2B >= 0) {
+    // one token per thread per round; B consecutive lanes own one block
 #pragma unroll 4
     for (int r = 0; r < kTileTok / kTileThreads; ++r) {
       const int64_t g = base + r * kTileThreads + tid;
@@ -169,7 +215,7 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
   __shared__ uint64_t s_carry[2];
   __shared__ long long s_red[kScanThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const PairDesc pd = p.pairs[blockIdx.x];
+  const PairDesc pd = p.pairs ? p.pairs[blockIdx.x] : p.inl[blockIdx.x];
   const int B = p.B;
   const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
   const int64_t lim = nbc < nbs ? nbc : nbs;                 // blocks that can be compared
@@ -233,7 +279,7 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
 
   // token-level first mismatch over this pair's tiles
   long long lcp = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
-  const int64_t t0 = pd.tile_off, t1 = p.pairs[blockIdx.x + 1].tile_off;
+  const int64_t t0 = pd.tile_off, t1 = p.pairs ? p.pairs[blockIdx.x + 1].tile_off : p.inl[blockIdx.x + 1].tile_off;
   for (int64_t t = t0 + tid; t < t1; t += kScanThreads) {
     long long v = p.tile_mis[t];
     lcp = v < lcp ? v : lcp;
@@ -276,9 +322,16 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
   if (n_pairs == 0) return TALARIA_OK;
   if (!cont_off || !sess_off) return TALARIA_ERR_INVALID_ARG;
-  DescSlot *slot;
-  TAL_TRY(acquire_slot(ctx, (size_t)(n_pairs + 1) * sizeof(PairDesc), &slot));
-  PairDesc *pd = (PairDesc *)slot->h;
+  // few pairs: descriptors ride in the kernel parameters (no upload); otherwise a
+  // pinned slot holds the pair table followed by one pair index per tile
+  const bool inl = n_pairs <= kInlinePairs;
+  PrefixParams p{};
+  std::vector<PairDesc> big;
+  PairDesc *pd = p.inl;
+  if (!inl) {
+    big.resize((size_t)n_pairs + 1);
+    pd = big.data();
+  }
   int64_t cb = 0, sb = 0, tiles = 0;
   for (int32_t q = 0; q < n_pairs; ++q) {
     int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
@@ -297,10 +350,19 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   const size_t dig_c_bytes = (size_t)cb * 8, dig_s_bytes = derive ? (size_t)sb * 8 : 0;
   const size_t need = dig_c_bytes + dig_s_bytes + (size_t)tiles * 8 + 64;
   TAL_TRY(grow(ctx, &ctx->prefix_scratch, need));
-  TAL_TRY(upload_slot(ctx, slot, (size_t)(n_pairs + 1) * sizeof(PairDesc), stream));
-
-  PrefixParams p{};
-  p.pairs = (const PairDesc *)slot->d;
+  DescSlot *slot = nullptr;
+  if (!inl) {
+    const size_t pair_bytes = ((size_t)(n_pairs + 1) * sizeof(PairDesc) + 15) & ~(size_t)15;
+    const size_t desc_bytes = pair_bytes + (size_t)tiles * sizeof(int32_t);
+    TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+    memcpy(slot->h, big.data(), (size_t)(n_pairs + 1) * sizeof(PairDesc));
+    int32_t *tp = (int32_t *)(slot->h + pair_bytes);
+    for (int32_t q = 0; q < n_pairs; ++q)
+      for (int64_t t = big[q].tile_off; t < big[q + 1].tile_off; ++t) tp[t] = q;
+    TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+    p.pairs = (const PairDesc *)slot->d;
+    p.tile_pair = (const int32_t *)(slot->d + pair_bytes);
+  }
   p.n_pairs = n_pairs;
   p.B = B;
   p.log2B = -1;
@@ -327,7 +389,7 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   prefix_chain_kernel<<<(unsigned)n_pairs, kScanThreads, 0, stream>>>(p);
   TAL_CUDA(ctx, cudaGetLastError());
   ctx->counters.kernel_launches++;
-  return release_slot(ctx, slot, stream);
+  return slot ? release_slot(ctx, slot, stream) : TALARIA_OK;
 }
 
 }  // namespace tal
