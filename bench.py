@@ -36,6 +36,18 @@ PCIE5_X16_GBS = 63.0          # 32 GT/s x 16 lanes x 128/130 / 8, per direction
 POOL_BLOCKS = 4096
 PREFIX_TOKENS, CONT_TOKENS, SHARED_TOKENS = 25_000, 27_000, 24_000
 STAGE_CHUNK = 2 << 20
+STAGE_FRACTION = 1.0
+# DRAM bytes per algorithmic byte of stage_copy_kernel, from the ncu capture summarised in
+# profiles/stage_copy_kernel_small.md (dram__bytes_read.sum + dram__bytes_write.sum over 2 x payload)
+STAGE_TRAFFIC_RATIO = 0.987
+
+
+def apply_scale(scale: str):
+    """'small' is the same step on a workload that fits an ncu capture: 1,024-block pool,
+    4,096-token session, the first 1/32 of the staging plan (about 5 GB on the device)."""
+    global POOL_BLOCKS, PREFIX_TOKENS, CONT_TOKENS, SHARED_TOKENS, STAGE_FRACTION
+    if scale == "small":
+        POOL_BLOCKS, PREFIX_TOKENS, CONT_TOKENS, SHARED_TOKENS, STAGE_FRACTION = 1024, 4096, 4608, 4000, 1 / 32
 
 
 def measured_peaks():
@@ -218,6 +230,9 @@ def run_gpu(args):
 
     ws = wl.moe_weight_set()
     plan, span = wl.stage_plan(ws.sizes, STAGE_CHUNK)
+    if STAGE_FRACTION < 1.0:
+        plan = plan[: max(1, int(len(plan) * STAGE_FRACTION))]
+        span = plan[-1][0] + plan[-1][1]
     if args.no_stage:
         plan, span = [], 0
     staging = torch.empty(max(span, 16), dtype=torch.uint8, device=dev)
@@ -329,7 +344,7 @@ def run_gpu(args):
         gs = wl.rng(2, 99)
         img_dev_view = image        # pinned host tensor
         for _ in range(64):
-            l, p, i = int(gs.integers(0, 94)), int(gs.integers(0, 2)), int(gs.integers(0, n))
+            l, p, i = int(gs.integers(0, shape.num_layers)), int(gs.integers(0, 2)), int(gs.integers(0, n))
             a = l * strides[0] + p * strides[1] + i * strides[2]
             chunk = img_dev_view[a:a + C]
             pl = planes[l * 2 + p].view(torch.uint8)
@@ -337,7 +352,7 @@ def run_gpu(args):
             if i < nr:
                 check &= bool(torch.equal(pl[int(bt2[i]) * C:(int(bt2[i]) + 1) * C].cpu(), chunk))
         r = d_res.cpu().numpy()
-        check &= [int(r[0]), int(r[1]), int(r[2]), int(r[3]) & 0xFFFFFFFF] == [SHARED_TOKENS, SHARED_TOKENS // 16, SHARED_TOKENS, 0]
+        check &= [int(r[0]), int(r[1]), int(r[2]), int(r[3]) & 0xFFFFFFFF] == [SHARED_TOKENS, SHARED_TOKENS // 16, SHARED_TOKENS // 16 * 16, 0]
         if len(plan_arr):
             for off, nb, _ in (plan[0], plan[len(plan) // 2], plan[-1]):
                 check &= bool(torch.equal(slots[off:off + nb], staging[off:off + nb]))
@@ -349,25 +364,29 @@ def run_gpu(args):
 
     peaks, peaks_kind = measured_peaks()
     hbm_peak = float(peaks["hbm_gbs"])
-    roof_link = {
-        "bound": "host_link", "kernel": "kv_restore + kv_offload (variant %d)" % variant_used,
-        "achieved": link_bytes / ((phase["offload"] + phase["restore"]) * 1e6),
-        "peak": (ceilings["h2d"] * res_bytes + ceilings["d2h"] * off_bytes) / link_bytes, "unit": "GB/s",
-        "peak_kind": "pinned cudaMemcpyAsync 1 GiB measured in this run (nominal PCIe Gen5 x16: 63.0 GB/s)",
-        "offload_gbs": off_bytes / (phase["offload"] * 1e6), "restore_gbs": res_bytes / (phase["restore"] * 1e6),
-        "ceiling_d2h_gbs": ceilings["d2h"], "ceiling_h2d_gbs": ceilings["h2d"],
-        "frac_of_nominal": link_bytes / ((phase["offload"] + phase["restore"]) * 1e6) / PCIE5_X16_GBS,
-        "traffic": None,
+    off_gbs, res_gbs = off_bytes / (phase["offload"] * 1e6), res_bytes / (phase["restore"] * 1e6)
+    link_ach = link_bytes / ((phase["offload"] + phase["restore"]) * 1e6)
+    link_peak = link_bytes / (res_bytes / ceilings["h2d"] + off_bytes / ceilings["d2h"])
+    host_link = {
+        "bound": "host_link", "op": "kv_offload + kv_restore (variant %d)" % variant_used,
+        "achieved": link_ach, "peak": link_peak, "unit": "GB/s", "frac": link_ach / link_peak,
+        "peak_kind": "pinned cudaMemcpyAsync, 1 GiB, best of 6, measured in this run",
+        "offload_gbs": off_gbs, "restore_gbs": res_gbs, "ceiling_d2h_gbs": ceilings["d2h"],
+        "ceiling_h2d_gbs": ceilings["h2d"], "offload_frac": off_gbs / ceilings["d2h"],
+        "restore_frac": res_gbs / ceilings["h2d"], "nominal_pcie5_x16_gbs": PCIE5_X16_GBS,
+        "frac_of_nominal": link_ach / PCIE5_X16_GBS,
     }
-    roof_link["frac"] = roof_link["achieved"] / roof_link["peak"]
-    roof_hbm = None
+    roofline = None
     if len(plan_arr):
         ach = 2 * stage_bytes / (phase["stage"] * 1e6)
-        roof_hbm = {"bound": "hbm", "kernel": "stage_copy_kernel", "achieved": ach, "peak": hbm_peak,
-                    "peak_kind": f"{peaks_kind} copy bandwidth (MEASURED_PEAKS.json)", "unit": "GB/s",
-                    "frac": ach / hbm_peak, "frac_of_nominal_8tbs": ach / 8000.0,
-                    "algorithmic_bytes": 2 * stage_bytes, "traffic": None,
-                    "note": "timed while the concurrent offload's bounce kernels and DMA share the GPU"}
+        roofline = {"bound": "hbm", "kernel": "stage_copy_kernel", "achieved": ach, "peak": hbm_peak,
+                    "unit": "GB/s", "frac": ach / hbm_peak,
+                    "peak_kind": f"hbm_gbs of {peaks_kind} (MEASURED_PEAKS.json copy bandwidth)",
+                    "frac_of_nominal_8tbs": ach / 8000.0, "algorithmic_bytes": 2 * stage_bytes,
+                    "traffic": (STAGE_TRAFFIC_RATIO * 2 * stage_bytes) if STAGE_TRAFFIC_RATIO else None,
+                    "launch_ms": phase["stage"],
+                    "note": "dominant kernel by GPU time; timed inside the step, where it shares the GPU "
+                            "with the concurrent offload's packing kernels and DMA"}
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -378,18 +397,19 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": "configs[1]: Qwen3-235B-shaped KV (94 layers x 4 KV heads x 128, bf16, 16-token "
-                               "blocks), one 25,000-token session: offload 1,563 blocks || stage 58.95 GB D2D, "
-                               "match 27,000-token continuation, restore 1,500 matched blocks",
+        "config": {"workload": ("configs[1]: " if args.scale == "full" else "profiling-sized cut of configs[1]: ") +
+                               "Qwen3-235B-shaped KV (94 layers x 4 KV heads x 128, bf16, 16-token blocks), one "
+                               f"{PREFIX_TOKENS:,}-token session: offload {n:,} blocks || stage {stage_bytes / 1e9:.2f} GB "
+                               f"D2D, match {CONT_TOKENS:,}-token continuation, restore {nr:,} matched blocks",
                    "pool_blocks": POOL_BLOCKS, "host_layout": "page-first", "stage_chunk_bytes": STAGE_CHUNK,
-                   "stage_bytes": stage_bytes, "variant": variant_used, "replicas": world,
+                   "stage_bytes": stage_bytes, "variant": variant_used, "replicas": world, "scale": args.scale,
                    "l2": "every op streams inputs far larger than the 126 MB L2 (4.8 GB / 59 GB)"},
         "phases_ms": phase, "self_check": check,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": res_bytes + (CONT_TOKENS + PREFIX_TOKENS) * 4 + (PREFIX_TOKENS // 16) * 8 + (n + nr) * 4,
                 "d2h_bytes_per_step": off_bytes + 32 + (CONT_TOKENS // 16) * 8},
         "gpu_launches": int(counters.kernel_launches), "copy_engine_copies": int(counters.memcpy_calls),
-        "roofline": roof_link, "roofline_hbm": roof_hbm, "cpu_baseline": cpu, "clocks": clocks,
+        "roofline": roofline, "host_link": host_link, "cpu_baseline": cpu, "clocks": clocks,
         "prefix_match": {"us_per_call": phase["match"] * 1e3,
                          "tokens_per_s": (CONT_TOKENS + PREFIX_TOKENS) / (phase["match"] * 1e-3)},
     }
@@ -405,10 +425,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 zero-copy, 2 bounce+DMA, 3 per-run DMA")
+    ap.add_argument("--scale", default="full", choices=["full", "small"], help="small = profiling-sized workload")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    apply_scale(args.scale)
     if args.impl == "reference":
         run_reference(args)
     else:
