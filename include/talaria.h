@@ -186,6 +186,42 @@ talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
                                            uint64_t seed, uint64_t *h_cont_hashes_out,
                                            talaria_match_t *h_results, void *stream);
 
+/* No counterpart in the paper: an allocation-free form of talaria_prefix_match.
+ *
+ * Who needs it: a serving process that has handed all of HBM to its own memory
+ * manager, or a latency-critical thread inside a serving loop.  Such callers must
+ * not reach the CUDA allocator: a device allocation may simply fail when no HBM is
+ * left, and allocating or freeing device memory makes every stream of the device
+ * wait.  They also may not want a talaria context, whose creation allocates.
+ *
+ * This entry point takes no context and allocates nothing, on the device or on the
+ * host: no cudaMalloc / cudaFree, no pinned staging, no copies.  Its scratch (block
+ * digests and per-tile mismatch positions) is a fixed 1 MiB array inside the library
+ * image, held by every GPU that loads the library until the process exits, and the
+ * pair descriptors travel in the kernel parameters.  Arguments and results are
+ * exactly those of talaria_prefix_match; the caller still owns every buffer.
+ *
+ * Limits (TALARIA_ERR_EXTENT beyond them, nothing is launched):
+ *   n_pairs <= 8, and
+ *   sum over pairs of floor(Tc/B) [+ floor(Ts/B) when d_sess_hashes is NULL]
+ *     + ceil(max(Tc,Ts)/2048)  <=  131,072 scratch words
+ *   (for example one pair of two 1,000,000-token streams at B = 16).
+ * The work runs on the CURRENT device (cudaSetDevice is the caller's business).
+ * The first call on each device looks up the scratch array's device address; make
+ * that first call before any stream capture.  All calls in a process share the one
+ * scratch array per device: two calls whose kernels can overlap on the GPU
+ * (different streams, no ordering between them) race on it and must be serialised
+ * by the caller.  The array keeps the previous call's contents; nothing in it
+ * needs clearing because every word that is read is written first in the same
+ * call. */
+talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const int32_t *d_cont_tokens,
+                                             const int64_t *cont_offsets,
+                                             const int32_t *d_sess_tokens,
+                                             const int64_t *sess_offsets,
+                                             const uint64_t *d_sess_hashes, int32_t block_tokens,
+                                             uint64_t seed, uint64_t *d_cont_hashes_out,
+                                             talaria_match_t *d_results, void *stream);
+
 /* App. B "Prefix agreement": the longest leading block range on which all R
  * ranks committed a block and hold the same chained hash.  Pure host arithmetic.
  * committed_blocks: HOST int64[R]; hashes: HOST uint64[R][stride]. */

@@ -102,6 +102,7 @@ _SIGNATURES = {
     "talaria_block_hash": (C.c_int32, [_P, _P, C.c_int64, C.c_int32, C.c_uint64, _P, _P]),
     "talaria_prefix_match": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
     "talaria_prefix_match_host": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
+    "talaria_prefix_match_static": (C.c_int32, [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
     "talaria_prefix_agree": (C.c_int64, [C.c_int32, _P, _P, C.c_int64]),
     "talaria_kv_offload": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_restore": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
@@ -242,6 +243,19 @@ class Talaria:
                                                     block_tokens, C.c_uint64(seed), _ptr(h_cont_hashes_out),
                                                     _ptr(h_results), _stream_ptr(stream)),
                     "talaria_prefix_match_host")
+
+    @staticmethod
+    def prefix_match_static(n_pairs: int, d_cont_tokens, cont_offsets, d_sess_tokens, sess_offsets,
+                            d_sess_hashes, block_tokens: int, seed: int, d_cont_hashes_out, d_results,
+                            stream=None):
+        """Allocation-free form of prefix_match: no context, fixed scratch inside the library,
+        at most 8 pairs.  Runs on the current CUDA device."""
+        co, so = _i64(cont_offsets), _i64(sess_offsets)
+        rc = lib().talaria_prefix_match_static(n_pairs, _ptr(d_cont_tokens), _ptr(co), _ptr(d_sess_tokens),
+                                               _ptr(so), _ptr(d_sess_hashes), block_tokens, C.c_uint64(seed),
+                                               _ptr(d_cont_hashes_out), _ptr(d_results), _stream_ptr(stream))
+        if rc != OK:
+            raise TalariaError(rc, "talaria_prefix_match_static")
 
     @staticmethod
     def prefix_agree(committed_blocks, hashes: np.ndarray) -> int:

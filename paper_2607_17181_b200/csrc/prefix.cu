@@ -475,3 +475,107 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
   TAL_CUDA(ctx, cudaStreamSynchronize(stream));
   return TALARIA_OK;
 }
+
+
+// ---------------------------------------------------------------------------
+// Prefix match without any allocation.
+//
+// Same two kernels as talaria_prefix_match, but the digests and per-tile mismatch
+// positions live in a fixed array that is part of the loaded library image, and
+// the pair descriptors travel in the kernel parameters.  Nothing is allocated on
+// the device or on the host, no context is needed, and no copy is issued.
+namespace tal {
+
+constexpr int64_t kStaticWords = 131072;   // 1 MiB of scratch: 8 bytes per block digest / tile
+static __device__ __align__(256) unsigned long long g_static_scratch[kStaticWords];
+
+constexpr int kStaticMaxDevices = 64;
+static std::mutex g_static_mu;
+static unsigned long long *g_static_addr[kStaticMaxDevices];   // device address, per device
+
+// The array's name is only a host-side handle here; the address a kernel can use has
+// to be asked for, once per device, with that device current.
+static talaria_status_t static_scratch_address(unsigned long long **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return TALARIA_ERR_CUDA;
+  }
+  if (dev < 0 || dev >= kStaticMaxDevices) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (!g_static_addr[dev]) {
+    void *ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      (void)cudaGetLastError();
+      return TALARIA_ERR_CUDA;
+    }
+    g_static_addr[dev] = (unsigned long long *)ptr;
+  }
+  *out = g_static_addr[dev];
+  return TALARIA_OK;
+}
+
+}  // namespace tal
+
+extern "C" talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const int32_t *d_cont_tokens,
+                                                        const int64_t *cont_offsets,
+                                                        const int32_t *d_sess_tokens,
+                                                        const int64_t *sess_offsets,
+                                                        const uint64_t *d_sess_hashes, int32_t block_tokens,
+                                                        uint64_t seed, uint64_t *d_cont_hashes_out,
+                                                        talaria_match_t *d_results, void *stream) {
+  const int32_t B = block_tokens;
+  if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_pairs == 0) return TALARIA_OK;
+  if (n_pairs > kInlinePairs) return TALARIA_ERR_EXTENT;
+  if (!cont_offsets || !sess_offsets || !d_results) return TALARIA_ERR_INVALID_ARG;
+  PrefixParams p{};
+  int64_t cb = 0, sb = 0, tiles = 0;
+  for (int32_t q = 0; q < n_pairs; ++q) {
+    const int64_t Tc = cont_offsets[q + 1] - cont_offsets[q], Ts = sess_offsets[q + 1] - sess_offsets[q];
+    if (Tc < 0 || Ts < 0 || cont_offsets[q] < 0 || sess_offsets[q] < 0) return TALARIA_ERR_INVALID_ARG;
+    p.inl[q] = PairDesc{cont_offsets[q], sess_offsets[q], Tc, Ts, cb, sb, tiles};
+    cb += Tc / B;
+    sb += Ts / B;
+    tiles += (std::max(Tc, Ts) + kTileTok - 1) / kTileTok;
+  }
+  p.inl[n_pairs] = PairDesc{cont_offsets[n_pairs], sess_offsets[n_pairs], 0, 0, cb, sb, tiles};
+  if (cont_offsets[n_pairs] > cont_offsets[0] && !d_cont_tokens) return TALARIA_ERR_INVALID_ARG;
+  if (sess_offsets[n_pairs] > sess_offsets[0] && !d_sess_tokens) return TALARIA_ERR_INVALID_ARG;
+  const bool derive = (d_sess_hashes == nullptr);
+  const int64_t words = cb + (derive ? sb : 0) + tiles;
+  if (words > kStaticWords) return TALARIA_ERR_EXTENT;   // beyond the built-in scratch
+  unsigned long long *scratch = nullptr;
+  TAL_TRY(static_scratch_address(&scratch));
+  p.pairs = nullptr;
+  p.tile_pair = nullptr;
+  p.n_pairs = n_pairs;
+  p.B = B;
+  p.log2B = -1;
+  if (B <= 32 && (B & (B - 1)) == 0) {
+    int l = 0;
+    while ((1 << l) < B) ++l;
+    p.log2B = l;
+  }
+  p.need_sess_digest = derive ? 1 : 0;
+  p.cont = d_cont_tokens;
+  p.sess = d_sess_tokens;
+  // Every word that is read is written earlier in the same call (digests of full
+  // blocks and one mismatch position per tile), so nothing has to start at zero.
+  p.dig_c = (uint64_t *)scratch;
+  p.dig_s = (uint64_t *)scratch + cb;
+  p.tile_mis = (long long *)(scratch + cb + (derive ? sb : 0));
+  p.sess_hashes = d_sess_hashes;
+  p.cont_hashes_out = d_cont_hashes_out;
+  p.results = d_results;
+  p.seed = seed;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (tiles > 0) {
+    prefix_tile_kernel<<<(unsigned)tiles, kTileThreads, 0, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return TALARIA_ERR_CUDA;
+  }
+  prefix_chain_kernel<<<(unsigned)n_pairs, kScanThreads, 0, st>>>(p);
+  if (cudaGetLastError() != cudaSuccess) return TALARIA_ERR_CUDA;
+  return TALARIA_OK;
+}
