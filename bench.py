@@ -195,6 +195,7 @@ def run_gpu(args):
     import torch
     import torch.distributed as dist
     from paper_2607_17181_b200 import binding as tb
+    from paper_2607_17181_b200.replicas import job_totals
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -314,11 +315,7 @@ def run_gpu(args):
             nr = step(e2e, True)
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms, _ = job_totals(e0.elapsed_time(e1), 0.0, dist if world > 1 else None, dev)
         return ms / args.steps, nr, ctx.get_counters()
 
     sampler = ClockSampler(local)
