@@ -46,8 +46,27 @@ __device__ __forceinline__ void decode_chunk(const KvCopyParams &p, int64_t w, i
   img_off = d0 * p.sd[0] + d1 * p.sd[1] + d2 * p.sd[2];
 }
 
+// 256-bit streaming accesses (sm_100): fewer instructions per byte than 128-bit ones.
+struct alignas(32) Vec32 {
+  unsigned r[8];
+};
+__device__ __forceinline__ Vec32 ld_cs_32(const void *p) {
+  Vec32 v;
+  asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]),
+                 "=r"(v.r[6]), "=r"(v.r[7])
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_cs_32(void *p, const Vec32 &v) {
+  asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]),
+               "r"(v.r[3]), "r"(v.r[4]), "r"(v.r[5]), "r"(v.r[6]), "r"(v.r[7]), "l"(p)
+               : "memory");
+}
+
 // TO_IMAGE: pool -> image (offload / gather); else image -> pool (restore / scatter).
-template <bool TO_IMAGE>
+// VB: bytes per access (16 or 32); every lane keeps 128 bytes in flight per step.
+template <bool TO_IMAGE, int VB>
 __global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant__ KvCopyParams p) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -62,18 +81,26 @@ __global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant_
     int64_t blk = p.table[i];
     char *pool = (char *)p.plane_base[lp] + blk * p.chunk_bytes + part * kPart;
     char *img = p.img + img_off + part * kPart;
-    const int4 *src = (const int4 *)(TO_IMAGE ? pool : img);
-    int4 *dst = (int4 *)(TO_IMAGE ? img : pool);
+    const char *src = TO_IMAGE ? pool : img;
+    char *dst = TO_IMAGE ? img : pool;
     int64_t left = p.chunk_bytes - part * kPart;
     if (left >= kPart) {
-      int4 v[8];
+      if (VB == 32) {
+        Vec32 v[4];
 #pragma unroll
-      for (int k = 0; k < 8; ++k) v[k] = __ldcs(src + lane + k * 32);
+        for (int k = 0; k < 4; ++k) v[k] = ld_cs_32(src + (lane + k * 32) * 32);
 #pragma unroll
-      for (int k = 0; k < 8; ++k) __stcs(dst + lane + k * 32, v[k]);
+        for (int k = 0; k < 4; ++k) st_cs_32(dst + (lane + k * 32) * 32, v[k]);
+      } else {
+        int4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = __ldcs((const int4 *)src + lane + k * 32);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) __stcs((int4 *)dst + lane + k * 32, v[k]);
+      }
     } else {
       int n16 = (int)(left >> 4);
-      for (int k = lane; k < n16; k += 32) __stcs(dst + k, __ldcs(src + k));
+      for (int k = lane; k < n16; k += 32) __stcs((int4 *)dst + k, __ldcs((const int4 *)src + k));
     }
   }
 }
@@ -107,7 +134,7 @@ struct Plan {
   int64_t L, P, n, C, chunks;
   ImgOrder ord;
   int64_t run_chunks;  // chunks that are contiguous in the image, aligned in w
-  bool vec;            // 16-byte path usable
+  int vec;             // widest usable access: 32, 16, or 0 (byte path)
 };
 
 static talaria_status_t make_plan(const talaria_kv_layout_t *kv, int64_t n, const void *img,
@@ -155,14 +182,14 @@ static talaria_status_t make_plan(const talaria_kv_layout_t *kv, int64_t n, cons
     bytes *= d[k].extent;
   }
   pl.run_chunks = run;
-  bool aligned = (pl.C % 16 == 0) && (((uintptr_t)img) % 16 == 0);
+  uintptr_t bits = (uintptr_t)pl.C | (uintptr_t)img;    // low bits of everything an address is built from
   for (int k = 0; k < 3; ++k)
-    if (d[k].extent != 1 && d[k].stride % 16 != 0) aligned = false;
+    if (d[k].extent != 1) bits |= (uintptr_t)d[k].stride;
   for (int64_t k = 0; k < pl.L * pl.P; ++k) {
     if (!kv->plane_base[k]) return TALARIA_ERR_INVALID_ARG;
-    if (((uintptr_t)kv->plane_base[k]) % 16 != 0) aligned = false;
+    bits |= (uintptr_t)kv->plane_base[k];
   }
-  pl.vec = aligned;
+  pl.vec = (bits % 32 == 0) ? 32 : (bits % 16 == 0) ? 16 : 0;
   *out = pl;
   return TALARIA_OK;
 }
@@ -196,21 +223,25 @@ static talaria_status_t validate_table(talaria_ctx *ctx, const talaria_kv_layout
   return TALARIA_OK;
 }
 
+// vec: access width the addresses allow (0 = byte path); img_bits: low bits of the image base in use.
 template <bool TO_IMAGE>
-static talaria_status_t launch_copy(talaria_ctx *ctx, const KvCopyParams &p, bool vec, int grid_cap,
+static talaria_status_t launch_copy(talaria_ctx *ctx, const KvCopyParams &p, int vec, int64_t grid_cap,
                                     cudaStream_t stream) {
   if (p.w1 <= p.w0) return TALARIA_OK;
+  if ((uintptr_t)p.img % 32 != 0 && vec == 32) vec = 16;
+  if ((uintptr_t)p.img % 16 != 0) vec = 0;
   if (vec) {
     const int threads = 512;
     int64_t parts = (p.chunk_bytes + kPart - 1) / kPart;
     int64_t warps = (p.w1 - p.w0) * parts;
     int64_t need = (warps + threads / 32 - 1) / (threads / 32);
     int grid = (int)std::max<int64_t>(1, std::min<int64_t>(need, grid_cap));
-    kv_copy_vec_kernel<TO_IMAGE><<<grid, threads, 0, stream>>>(p);
+    if (vec == 32) kv_copy_vec_kernel<TO_IMAGE, 32><<<grid, threads, 0, stream>>>(p);
+    else           kv_copy_vec_kernel<TO_IMAGE, 16><<<grid, threads, 0, stream>>>(p);
   } else {
     const int threads = 256;
     int64_t need = ((p.w1 - p.w0) + threads / 32 - 1) / (threads / 32);
-    int grid = (int)std::max<int64_t>(1, std::min<int64_t>(need, grid_cap));
+    int grid = (int)std::max<int64_t>(1, std::min<int64_t>(need, std::min<int64_t>(grid_cap, 1 << 20)));
     kv_copy_byte_kernel<TO_IMAGE><<<grid, threads, 0, stream>>>(p);
   }
   TAL_CUDA(ctx, cudaGetLastError());
@@ -218,8 +249,8 @@ static talaria_status_t launch_copy(talaria_ctx *ctx, const KvCopyParams &p, boo
   return TALARIA_OK;
 }
 
-static talaria_status_t launch_dir(talaria_ctx *ctx, bool to_image, const KvCopyParams &p, bool vec,
-                                   int grid_cap, cudaStream_t stream) {
+static talaria_status_t launch_dir(talaria_ctx *ctx, bool to_image, const KvCopyParams &p, int vec,
+                                   int64_t grid_cap, cudaStream_t stream) {
   return to_image ? launch_copy<true>(ctx, p, vec, grid_cap, stream)
                   : launch_copy<false>(ctx, p, vec, grid_cap, stream);
 }
@@ -230,7 +261,14 @@ static void set_image_strides(KvCopyParams &p, const ImgOrder &o, int64_t sL, in
   p.sd[o.pos_i] = sI;
 }
 
-static int zc_grid(const talaria_ctx *ctx) { return ctx->cfg.zc_ctas > 0 ? ctx->cfg.zc_ctas : 32; }
+// Zero-copy kernels are bound by the host link: 8 CTAs already saturate it, 32 leave headroom
+// and keep 100+ SMs free for whatever else is running.
+static int64_t zc_grid(const talaria_ctx *ctx) { return ctx->cfg.zc_ctas > 0 ? ctx->cfg.zc_ctas : 32; }
+// Pack / unpack kernels of the bounce variant only have to stay ahead of a 56 GB/s copy engine;
+// a small grid does that with a 20x margin and barely disturbs concurrent kernels.
+static int64_t pack_grid(const talaria_ctx *ctx) { return 2 * zc_grid(ctx); }
+// In-HBM gather / scatter: one short CTA per 16 warps of work, scheduled by the hardware.
+static int64_t full_grid() { return 0x7fffffff; }
 
 // Number of runs of adjacent ids in a table (bt[i+1] == bt[i]+1 continues a run).
 static int64_t count_id_runs(const int32_t *bt, int64_t n) {
@@ -257,7 +295,7 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
     TAL_TRY(require_device_pointer(ctx, img));
   } else {
     TAL_TRY(mapped_pointer(ctx, img, &img_dev));
-    if (((uintptr_t)img_dev) % 16 != 0) pl.vec = false;
+    if (((uintptr_t)img_dev) % 16 != 0) pl.vec = 0;
   }
 
   // descriptor: plane pointers, then the table slice
@@ -283,7 +321,7 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
     p.img = (char *)img_dev;
     set_image_strides(p, pl.ord, hl->stride_layer, hl->stride_plane, hl->stride_block);
     p.w0 = 0; p.w1 = pl.chunks;
-    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, hbm_grid(ctx, 512), stream));
+    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, full_grid(), stream));
     return release_slot(ctx, slot, stream);
   }
 
@@ -354,7 +392,7 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
     char *half = ln.buf + (size_t)j * ln.half;
     p.img = half - w0 * pl.C;   // so that offset(w) lands at (w - w0)*C inside the half
     p.w0 = w0; p.w1 = w1;
-    if (to_image) TAL_TRY(launch_dir(ctx, true, p, pl.vec && ((uintptr_t)half % 16 == 0), hbm_grid(ctx, 512), ln.s[j]));
+    if (to_image) TAL_TRY(launch_dir(ctx, true, p, pl.vec, pack_grid(ctx), ln.s[j]));
     for (int64_t ws = w0; ws < w1;) {
       int64_t we = std::min(w1, (ws / pl.run_chunks + 1) * pl.run_chunks);
       char *h = (char *)img + image_offset(pl, hl, ws);
@@ -365,7 +403,7 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
       ctx->counters.memcpy_calls++;
       ws = we;
     }
-    if (!to_image) TAL_TRY(launch_dir(ctx, false, p, pl.vec && ((uintptr_t)half % 16 == 0), hbm_grid(ctx, 512), ln.s[j]));
+    if (!to_image) TAL_TRY(launch_dir(ctx, false, p, pl.vec, pack_grid(ctx), ln.s[j]));
   }
   for (int j = 0; j < 2; ++j) {
     TAL_CUDA(ctx, cudaEventRecord(ln.done[j], ln.s[j]));

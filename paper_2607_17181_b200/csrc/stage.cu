@@ -3,9 +3,9 @@
 // pinned host copy (App. D: "reloads those chunks from host rather than copying
 // unsafe D2D sources").
 //
-// The D2D leg is one kernel over the whole plan: the plan is cut into 32 KiB tiles
+// The D2D leg is one kernel over the whole plan: the plan is cut into 64 KiB tiles
 // and every CTA takes one short contiguous span of tiles (512 KiB), moving each
-// tile with four 16-byte loads per thread in flight.  The grid is NOT persistent
+// tile with four 256-bit loads per thread in flight (128 bytes per thread).  The grid is NOT persistent
 // on purpose: staging runs next to KV offload / restore on other streams, and
 // short CTAs let the hardware scheduler interleave those kernels instead of
 // making them wait for a resident grid to drain.  The host precomputes the plan
@@ -27,8 +27,25 @@ struct StageEntry {
 };
 
 constexpr int kStageThreads = 512;
-constexpr int kStageTile = kStageThreads * 16 * 4;   // 32 KiB
-constexpr int kSpanTiles = 16;                       // tiles per CTA (512 KiB)
+constexpr int kStageTile = kStageThreads * 128;      // 64 KiB: 128 bytes in flight per thread
+constexpr int kSpanTiles = 8;                        // tiles per CTA (512 KiB)
+
+struct alignas(32) Vec32 {
+  unsigned r[8];
+};
+__device__ __forceinline__ Vec32 ld_cs_32(const void *p) {
+  Vec32 v;
+  asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]),
+                 "=r"(v.r[6]), "=r"(v.r[7])
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_cs_32(void *p, const Vec32 &v) {
+  asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]),
+               "r"(v.r[3]), "r"(v.r[4]), "r"(v.r[5]), "r"(v.r[6]), "r"(v.r[7]), "l"(p)
+               : "memory");
+}
 
 struct StageParams {
   const StageEntry *entries;   // DEVICE [n + 1]; entries[n].tile0 = total tiles
@@ -54,15 +71,23 @@ __global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_
     const int64_t len = min((int64_t)kStageTile, cur.bytes - off);
     const char *src = cur.src + off;
     char *dst = cur.dst + off;
-    if ((((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {
+    const uintptr_t low = (uintptr_t)src | (uintptr_t)dst;
+    if ((low & 31) == 0 && len == kStageTile) {
+      // full tile, 32-byte aligned: four 256-bit loads per thread in flight
+      Vec32 v[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) v[k] = ld_cs_32(src + ((size_t)tid + k * kStageThreads) * 32);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) st_cs_32(dst + ((size_t)tid + k * kStageThreads) * 32, v[k]);
+    } else if ((low & 15) == 0) {
       const int4 *s4 = (const int4 *)src;
       int4 *d4 = (int4 *)dst;
       if (len == kStageTile) {
-        int4 v[4];
+        int4 v[8];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) v[k] = __ldcs(s4 + tid + k * kStageThreads);
+        for (int k = 0; k < 8; ++k) v[k] = __ldcs(s4 + tid + k * kStageThreads);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) __stcs(d4 + tid + k * kStageThreads, v[k]);
+        for (int k = 0; k < 8; ++k) __stcs(d4 + tid + k * kStageThreads, v[k]);
       } else {
         const int n16 = (int)(len >> 4);
         for (int k = tid; k < n16; k += kStageThreads) __stcs(d4 + k, __ldcs(s4 + k));
