@@ -327,6 +327,24 @@ def run_gpu(args):
     variant_used = int(counters.last_variant)
     ms_e2e, _, _ = timed(True)
 
+    # ---- in-HBM block gather / scatter of the same session (outside the step; the metric's
+    # "gather GB/s vs HBM peak"): image in device memory, read + write bytes = 2 x payload
+    d_image = torch.empty(n * shape.bytes_per_block, dtype=torch.uint8, device=dev)
+    gather_ms = {}
+    for name, fn in (("gather", lambda: ctx.kv_gather(kv, bt, 0, n, d_image, hl)),
+                     ("scatter", lambda: ctx.kv_scatter(kv, bt2, 0, n, d_image, hl))):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        g0, g1 = ev(), ev()
+        g0.record()
+        for _ in range(5):
+            fn()
+        g1.record()
+        torch.cuda.synchronize()
+        gather_ms[name] = g0.elapsed_time(g1) / 5
+    del d_image
+
     off_bytes, res_bytes = n * shape.bytes_per_block, nr * shape.bytes_per_block
     link_bytes = off_bytes + res_bytes
     value = world * link_bytes / (ms_step * 1e6)
@@ -406,7 +424,13 @@ def run_gpu(args):
                 "h2d_bytes_per_step": res_bytes + (CONT_TOKENS + PREFIX_TOKENS) * 4 + (PREFIX_TOKENS // 16) * 8 + (n + nr) * 4,
                 "d2h_bytes_per_step": off_bytes + 32 + (CONT_TOKENS // 16) * 8},
         "gpu_launches": int(counters.kernel_launches), "copy_engine_copies": int(counters.memcpy_calls),
-        "roofline": roofline, "host_link": host_link, "cpu_baseline": cpu, "clocks": clocks,
+        "roofline": roofline, "host_link": host_link,
+        "hbm_gather": {"bound": "hbm", "kernel": "kv_copy_vec_kernel (talaria_kv_gather / talaria_kv_scatter)",
+                       "gather_gbs": 2 * off_bytes / (gather_ms["gather"] * 1e6),
+                       "scatter_gbs": 2 * off_bytes / (gather_ms["scatter"] * 1e6), "peak": hbm_peak, "unit": "GB/s",
+                       "frac": 2 * off_bytes / (gather_ms["gather"] * 1e6) / hbm_peak,
+                       "algorithmic_bytes": 2 * off_bytes, "timed": "alone, after the timed steps, 5 launches"},
+        "cpu_baseline": cpu, "clocks": clocks,
         "prefix_match": {"us_per_call": phase["match"] * 1e3,
                          "tokens_per_s": (CONT_TOKENS + PREFIX_TOKENS) / (phase["match"] * 1e-3)},
     }
