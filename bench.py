@@ -37,8 +37,8 @@ POOL_BLOCKS = 4096
 PREFIX_TOKENS, CONT_TOKENS, SHARED_TOKENS = 25_000, 27_000, 24_000
 STAGE_CHUNK = 2 << 20
 STAGE_FRACTION = 1.0
-# DRAM bytes per algorithmic byte of stage_copy_kernel, from the ncu capture summarised in
-# profiles/stage_copy_kernel_small.md (dram__bytes_read.sum + dram__bytes_write.sum over 2 x payload)
+# DRAM bytes per algorithmic byte of stage_copy_kernel, from an ncu capture of the profiling-sized
+# case (--scale small): (dram__bytes_read.sum + dram__bytes_write.sum) / (2 x payload)
 STAGE_TRAFFIC_RATIO = 0.987
 
 

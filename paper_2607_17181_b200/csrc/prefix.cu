@@ -215,6 +215,9 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
   __shared__ uint64_t s_carry[2];
   __shared__ long long s_red[kScanThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  // Launched as a programmatic dependent of the tile kernel: CTAs may be resident early,
+  // and this wait returns once the tile kernel has finished and its writes are visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const PairDesc pd = p.pairs ? p.pairs[blockIdx.x] : p.inl[blockIdx.x];
   const int B = p.B;
   const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
@@ -313,6 +316,22 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
   }
 }
 
+// The chain kernel is launched with programmatic stream serialization so its launch latency
+// overlaps the tile kernel; it blocks in griddepcontrol.wait until the tile kernel is done.
+static cudaError_t launch_chain(const PrefixParams &p, int n_pairs, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)n_pairs);
+  cfg.blockDim = dim3(kScanThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, prefix_chain_kernel, p);
+}
+
 // Host side: validates offsets, builds the pair table, sizes scratch, launches.
 static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont,
                                       const int64_t *cont_off, const int32_t *d_sess,
@@ -386,8 +405,7 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     TAL_CUDA(ctx, cudaGetLastError());
     ctx->counters.kernel_launches++;
   }
-  prefix_chain_kernel<<<(unsigned)n_pairs, kScanThreads, 0, stream>>>(p);
-  TAL_CUDA(ctx, cudaGetLastError());
+  TAL_CUDA(ctx, launch_chain(p, n_pairs, stream));
   ctx->counters.kernel_launches++;
   return slot ? release_slot(ctx, slot, stream) : TALARIA_OK;
 }
@@ -575,7 +593,9 @@ extern "C" talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const i
     prefix_tile_kernel<<<(unsigned)tiles, kTileThreads, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return TALARIA_ERR_CUDA;
   }
-  prefix_chain_kernel<<<(unsigned)n_pairs, kScanThreads, 0, st>>>(p);
-  if (cudaGetLastError() != cudaSuccess) return TALARIA_ERR_CUDA;
+  if (launch_chain(p, n_pairs, st) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return TALARIA_ERR_CUDA;
+  }
   return TALARIA_OK;
 }
