@@ -250,6 +250,24 @@ talaria_status_t talaria_kv_restore(talaria_ctx *ctx, const talaria_kv_layout_t 
                                     int64_t n_blocks, const void *host_src,
                                     const talaria_host_layout_t *hl, void *stream);
 
+/* The same restore, delivered layer by layer (App. C: the layer-first view matches the
+ * device-side layout used by attention kernels; Sec. 3.4 charges the restore to the
+ * prefill budget, so prefill of layer l should start as soon as layer l has landed).
+ * The result in the pool is exactly that of talaria_kv_restore.  In addition
+ * layer_events[l] (HOST array of num_layers cudaEvent_t handles created by the
+ * caller, passed as void*) is recorded once every chunk of layer l, both planes, is
+ * in the pool; a consumer stream calls cudaStreamWaitEvent on it.  Layers complete in
+ * increasing order for large images (copy-engine path, any host layout: contiguous or
+ * pitched transfers per layer); for small images, zero-copy contexts or layouts with
+ * neither planes nor blocks adjacent, all events are recorded after one ordinary
+ * restore.  Work enqueued on `stream` after the call still waits for the whole
+ * restore. */
+talaria_status_t talaria_kv_restore_layered(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                            const int32_t *new_block_table, int64_t first_block,
+                                            int64_t n_blocks, const void *host_src,
+                                            const talaria_host_layout_t *hl,
+                                            void *const *layer_events, void *stream);
+
 /* Several sessions in one call (one fused launch per variant where possible). */
 typedef struct {
   const int32_t *block_table; /* HOST */

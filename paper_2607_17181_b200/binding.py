@@ -106,6 +106,7 @@ _SIGNATURES = {
     "talaria_prefix_agree": (C.c_int64, [C.c_int32, _P, _P, C.c_int64]),
     "talaria_kv_offload": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_restore": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
+    "talaria_kv_restore_layered": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P, _P]),
     "talaria_kv_gather": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_scatter": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_offload_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
@@ -274,6 +275,16 @@ class Talaria:
 
     def kv_restore(self, kv, new_block_table, first_block, n_blocks, host_src, hl, stream=None):
         self._kv(lib().talaria_kv_restore, "talaria_kv_restore", kv, new_block_table, first_block, n_blocks, host_src, hl, stream)
+
+    def kv_restore_layered(self, kv, new_block_table, first_block, n_blocks, host_src, hl, layer_events, stream=None):
+        """layer_events: one torch.cuda.Event (already recorded once, so its handle exists) or raw
+        cudaEvent_t address per layer."""
+        bt = _i32(new_block_table)
+        handles = [e if isinstance(e, int) else e.cuda_event for e in layer_events]
+        arr = (C.c_void_p * len(handles))(*handles)
+        self._check(lib().talaria_kv_restore_layered(self._h, C.byref(kv), _ptr(bt), first_block, n_blocks,
+                                                     _ptr(host_src), C.byref(hl), arr, _stream_ptr(stream)),
+                    "talaria_kv_restore_layered")
 
     def kv_gather(self, kv, block_table, first_block, n_blocks, d_image, il, stream=None):
         self._kv(lib().talaria_kv_gather, "talaria_kv_gather", kv, block_table, first_block, n_blocks, d_image, il, stream)

@@ -412,6 +412,133 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
   return release_slot(ctx, slot, stream);
 }
 
+
+// ---------------------------------------------------------------------------
+// Layer-ordered restore (App. C: the layer-first view "matches the device-side KV
+// cache layout used by attention kernels"): the image is brought in layer by
+// layer, whatever its host layout, and an event per layer tells a consumer
+// (prefill of that layer) that the layer's K and V are in the pool.  Copy-engine
+// transfers (1-D or pitched 2-D, one per layer and piece) land in a bounce half;
+// the unpack kernel scatters it; the two halves alternate on two internal streams.
+static talaria_status_t kv_restore_layered(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                           const int32_t *table, int64_t first, int64_t n, const void *img,
+                                           const talaria_host_layout_t *hl, void *const *layer_events,
+                                           cudaStream_t stream) {
+  if (!kv || !hl || first < 0 || n < 0 || !layer_events) return TALARIA_ERR_INVALID_ARG;
+  if (kv->num_layers <= 0) return TALARIA_ERR_INVALID_ARG;
+  for (int32_t l = 0; l < kv->num_layers; ++l)
+    if (!layer_events[l]) return TALARIA_ERR_INVALID_ARG;
+  auto record_all = [&]() -> talaria_status_t {
+    for (int32_t l = 0; l < kv->num_layers; ++l) TAL_CUDA(ctx, cudaEventRecord((cudaEvent_t)layer_events[l], stream));
+    return TALARIA_OK;
+  };
+  if (n == 0) return record_all();
+  if (!table || !img) return TALARIA_ERR_INVALID_ARG;
+  Plan pl;
+  TAL_TRY(make_plan(kv, n, img, hl, &pl));
+  BounceLane &ln = ctx->lane[1];
+  const int64_t C = pl.C, P = pl.P, L = pl.L;
+  const int64_t sL = hl->stride_layer, sP = hl->stride_plane, sI = hl->stride_block;
+  const int64_t payload = pl.chunks * C, dma_min = ctx->cfg.dma_min_bytes > 0 ? ctx->cfg.dma_min_bytes : (8ll << 20);
+  const int64_t max_pitch = 1ll << 30;
+  // rows the copy engine can move: planes adjacent (a row per block) or blocks adjacent (a row per plane)
+  const bool rows_by_block = (P == 1 || sP == C);
+  const bool rows_by_plane = !rows_by_block && (n == 1 || sI == C);
+  const bool dma_ok = pl.vec != 0 && (int64_t)ln.half >= P * C && (rows_by_block || rows_by_plane) &&
+                      sI < max_pitch && sP < max_pitch && ctx->cfg.variant != TALARIA_VARIANT_ZEROCOPY &&
+                      (payload >= dma_min || ctx->cfg.variant == TALARIA_VARIANT_BOUNCE);
+  if (!dma_ok) {
+    // small or oddly laid out images: the ordinary restore, then every layer is ready at once
+    TAL_TRY(kv_transfer(ctx, kv, table, first, n, (void *)img, hl, stream, false, false));
+    return record_all();
+  }
+  const int32_t *bt = table + first;
+  TAL_TRY(validate_table(ctx, kv, bt, n, /*reject_dups=*/true));
+  void *alias;
+  TAL_TRY(mapped_pointer(ctx, img, &alias));
+
+  const size_t ptr_bytes = (size_t)(L * P) * sizeof(void *);
+  const size_t desc_bytes = ptr_bytes + (size_t)n * sizeof(int32_t);
+  DescSlot *slot;
+  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+  memcpy(slot->h, kv->plane_base, ptr_bytes);
+  memcpy(slot->h + ptr_bytes, bt, (size_t)n * sizeof(int32_t));
+  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+  ctx->counters.payload_bytes += payload;
+  ctx->counters.last_variant = TALARIA_VARIANT_BOUNCE;
+
+  // pieces: whole layers while a layer fits a bounce half, else block ranges of one layer
+  const int64_t layer_bytes = P * n * C;
+  const int64_t layers_per_piece = std::max<int64_t>(1, (int64_t)ln.half / layer_bytes);
+  const int64_t blocks_per_piece = layer_bytes <= (int64_t)ln.half ? n : std::max<int64_t>(1, (int64_t)ln.half / (P * C));
+
+  TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
+  for (int j = 0; j < 2; ++j) TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[j], ln.fork, 0));
+  int k = 0;
+  for (int64_t l0 = 0; l0 < L;) {
+    const int64_t l1 = (blocks_per_piece == n) ? std::min(L, l0 + layers_per_piece) : l0 + 1;
+    for (int64_t i0 = 0; i0 < n; i0 += blocks_per_piece, ++k) {
+      const int64_t i1 = std::min(n, i0 + blocks_per_piece), nn = i1 - i0, LL = l1 - l0;
+      const int j = k & 1;
+      char *half = ln.buf + (size_t)j * ln.half;
+      // host -> bounce half, one transfer per layer
+      for (int64_t l = l0; l < l1; ++l) {
+        const char *src = (const char *)img + l * sL + i0 * sI;
+        char *dst = half + (l - l0) * P * nn * C;
+        if (rows_by_block) {
+          if (nn == 1 || sI == P * C) {
+            TAL_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(nn * P * C), cudaMemcpyHostToDevice, ln.s[j]));
+          } else {
+            TAL_CUDA(ctx, cudaMemcpy2DAsync(dst, (size_t)(P * C), src, (size_t)sI, (size_t)(P * C), (size_t)nn,
+                                            cudaMemcpyHostToDevice, ln.s[j]));
+          }
+        } else {
+          if (P == 1 || sP == nn * C) {
+            TAL_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(P * nn * C), cudaMemcpyHostToDevice, ln.s[j]));
+          } else {
+            TAL_CUDA(ctx, cudaMemcpy2DAsync(dst, (size_t)(nn * C), src, (size_t)sP, (size_t)(nn * C), (size_t)P,
+                                            cudaMemcpyHostToDevice, ln.s[j]));
+          }
+        }
+        ctx->counters.memcpy_calls++;
+      }
+      // bounce half -> pool: the half holds [layer][block][plane] or [layer][plane][block]
+      KvCopyParams p{};
+      p.plane_base = (const void *const *)slot->d + l0 * P;
+      p.table = (const int32_t *)(slot->d + ptr_bytes) + i0;
+      p.chunk_bytes = C;
+      p.P = (int32_t)P;
+      p.img = half;
+      p.w0 = 0;
+      p.w1 = LL * P * nn;
+      if (rows_by_block) {        // digits: plane, block, layer
+        p.ord.e0 = P; p.ord.e1 = nn;
+        p.ord.lp_coef[0] = 1; p.ord.lp_coef[1] = 0; p.ord.lp_coef[2] = (int32_t)P;
+        p.ord.i_coef[0] = 0; p.ord.i_coef[1] = 1; p.ord.i_coef[2] = 0;
+        p.sd[0] = C; p.sd[1] = P * C; p.sd[2] = nn * P * C;
+      } else {                    // digits: block, plane, layer
+        p.ord.e0 = nn; p.ord.e1 = P;
+        p.ord.lp_coef[0] = 0; p.ord.lp_coef[1] = 1; p.ord.lp_coef[2] = (int32_t)P;
+        p.ord.i_coef[0] = 1; p.ord.i_coef[1] = 0; p.ord.i_coef[2] = 0;
+        p.sd[0] = C; p.sd[1] = nn * C; p.sd[2] = P * nn * C;
+      }
+      TAL_TRY(launch_dir(ctx, false, p, pl.vec, pack_grid(ctx), ln.s[j]));
+      TAL_CUDA(ctx, cudaEventRecord(ln.done[j], ln.s[j]));
+      if (i1 == n) {
+        // the layers of this piece are complete once the other half's earlier pieces are too
+        if (blocks_per_piece != n && k > 0) TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[j], ln.done[1 - j], 0));
+        for (int64_t l = l0; l < l1; ++l) TAL_CUDA(ctx, cudaEventRecord((cudaEvent_t)layer_events[l], ln.s[j]));
+      }
+    }
+    l0 = l1;
+  }
+  for (int j = 0; j < 2; ++j) {
+    TAL_CUDA(ctx, cudaEventRecord(ln.done[j], ln.s[j]));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[j], 0));
+  }
+  return release_slot(ctx, slot, stream);
+}
+
 }  // namespace tal
 
 using namespace tal;
@@ -437,6 +564,16 @@ extern "C" talaria_status_t talaria_kv_restore(talaria_ctx *ctx, const talaria_k
   TAL_ENTER(ctx);
   return kv_transfer(ctx, kv, new_block_table, first_block, n_blocks, (void *)host_src, hl,
                      (cudaStream_t)stream, false, false);
+}
+
+extern "C" talaria_status_t talaria_kv_restore_layered(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                                       const int32_t *new_block_table, int64_t first_block,
+                                                       int64_t n_blocks, const void *host_src,
+                                                       const talaria_host_layout_t *hl,
+                                                       void *const *layer_events, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_restore_layered(ctx, kv, new_block_table, first_block, n_blocks, host_src, hl, layer_events,
+                            (cudaStream_t)stream);
 }
 
 extern "C" talaria_status_t talaria_kv_gather(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
