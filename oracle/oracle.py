@@ -92,6 +92,11 @@ def lib():
                           C.POINTER(_HostLayout)]
         _lib.orc_stage.restype = C.c_int32
         _lib.orc_stage.argtypes = [C.POINTER(_Copy), C.c_int64, C.c_void_p, C.POINTER(_StageStats)]
+        _lib.orc_prestage.restype = C.c_int32
+        _lib.orc_prestage.argtypes = [C.POINTER(_Copy), C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.POINTER(_StageStats)]
+        _lib.orc_mark_dirty.restype = C.c_int64
+        _lib.orc_mark_dirty.argtypes = [C.POINTER(_Copy), C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         _lib.orc_stage_validate.restype = C.c_int32
         _lib.orc_stage_validate.argtypes = [C.POINTER(_Copy), C.c_int64, C.c_void_p]
     return _lib
@@ -278,3 +283,23 @@ def stage_validate(staging, hostcopy, slots, plan, dirty_bitmap) -> bool:
     arr = _plan_array(staging, hostcopy, slots, plan)
     bm = None if dirty_bitmap is None else np.ascontiguousarray(dirty_bitmap, dtype=np.uint8)
     return bool(lib().orc_stage_validate(arr, len(plan), _ptr(bm)))
+
+
+def prestage(staging: np.ndarray, hostcopy: np.ndarray, plan, blocked: Optional[np.ndarray],
+             staged: np.ndarray, dirty: np.ndarray) -> StageStats:
+    """plan: (staging_off, host_off, dst_off(unused), nbytes, chunk_id); staging is written;
+    staged / dirty bitmaps (uint8, LSB-first) are updated in place."""
+    arr = _plan_array(staging, hostcopy, staging, plan)
+    bl = None if blocked is None else np.ascontiguousarray(blocked, dtype=np.uint8)
+    st = _StageStats()
+    rc = lib().orc_prestage(arr, len(plan), _ptr(bl), _ptr(staged), _ptr(dirty), C.byref(st))
+    if rc != 0:
+        raise ValueError(f"orc_prestage rc={rc}")
+    return StageStats(st.d2d_bytes, st.h2d_bytes, st.dirty_chunks, st.missing_chunks)
+
+
+def mark_dirty(staging: np.ndarray, plan, alloc_off: int, alloc_bytes: int, staged: Optional[np.ndarray],
+               dirty: np.ndarray) -> int:
+    arr = _plan_array(staging, None, staging, plan)
+    return int(lib().orc_mark_dirty(arr, len(plan), staging.ctypes.data + alloc_off, alloc_bytes,
+                                    _ptr(staged), _ptr(dirty)))

@@ -20,6 +20,9 @@
  *                                   numpy slice cross-check, corrupted-dirty
  *                                   staging test)
  *   orc_prefix_agree      pinned   (App. B "Prefix agreement": brute force)
+ *   orc_prestage /
+ *   orc_mark_dirty        pinned   (Sec. 4.4 pre-staging protocol: numpy slice and
+ *                                   interval brute force)
  *   orc_block_hash        PARITY UNPINNED against the paper: Sec. 4.3 only says
  *                                   "cumulative prefix hash" per block and
  *                                   prints no function, width or value.  The
@@ -337,4 +340,58 @@ int32_t orc_stage_validate(const orc_copy_t *plan, int64_t n, const uint8_t *dir
         }
     }
     return 1;
+}
+
+/* ------------------------------------------------------------------ */
+/* Pre-staging while the current model serves (Sec. 4.4)                */
+/* ------------------------------------------------------------------ */
+
+static void orc_set_bit(uint8_t *bm, int64_t i, int v)
+{
+    if (v) bm[i >> 3] |= (uint8_t)(1u << (i & 7));
+    else   bm[i >> 3] &= (uint8_t)~(1u << (i & 7));
+}
+
+/* "The staging manager writes weights into fixed-size chunks": for every plan entry
+ * whose staging rows are not blocked (bit chunk_id of `blocked`: the rows currently
+ * belong to a KV allocation), copy the authoritative host bytes into the chunk's
+ * place in the staging region (src_dev), set its staged bit and clear its dirty
+ * bit.  Blocked chunks are left alone and stay unstaged.
+ * stats: h2d_bytes = bytes written, missing_chunks = chunks skipped,
+ *        dirty_chunks = dirty bits cleared by a rewrite, d2d_bytes = 0. */
+int32_t orc_prestage(const orc_copy_t *plan, int64_t n, const uint8_t *blocked, uint8_t *staged,
+                     uint8_t *dirty, orc_stage_stats_t *st)
+{
+    orc_stage_stats_t s = {0, 0, 0, 0};
+    for (int64_t k = 0; k < n; ++k) {
+        const orc_copy_t *c = &plan[k];
+        if (c->bytes < 0 || c->chunk_id < 0 || !c->src_dev || !c->src_host) return -1;
+        if (blocked && orc_bit(blocked, c->chunk_id)) { s.missing_chunks += 1; continue; }
+        memcpy((uint8_t *)c->src_dev, c->src_host, (size_t)c->bytes);
+        s.h2d_bytes += c->bytes;
+        if (staged) orc_set_bit(staged, c->chunk_id, 1);
+        if (dirty && orc_bit(dirty, c->chunk_id)) { orc_set_bit(dirty, c->chunk_id, 0); s.dirty_chunks += 1; }
+    }
+    if (st) *st = s;
+    return 0;
+}
+
+/* "marks a chunk dirty if a concurrent prefill allocation takes rows that overlap the
+ * chunk's staging range": every STAGED chunk whose staging bytes [src_dev, +bytes)
+ * intersect the allocation [alloc_base, +alloc_bytes) gets its dirty bit set.
+ * Returns how many bits changed from clean to dirty. */
+int64_t orc_mark_dirty(const orc_copy_t *plan, int64_t n, const uint8_t *alloc_base, int64_t alloc_bytes,
+                       const uint8_t *staged, uint8_t *dirty)
+{
+    int64_t changed = 0;
+    if (alloc_bytes <= 0) return 0;
+    for (int64_t k = 0; k < n; ++k) {
+        const orc_copy_t *c = &plan[k];
+        if (c->bytes <= 0 || c->chunk_id < 0 || !c->src_dev) continue;
+        if (staged && !orc_bit(staged, c->chunk_id)) continue;
+        if (c->src_dev < alloc_base + alloc_bytes && alloc_base < c->src_dev + c->bytes) {
+            if (!orc_bit(dirty, c->chunk_id)) { orc_set_bit(dirty, c->chunk_id, 1); changed += 1; }
+        }
+    }
+    return changed;
 }

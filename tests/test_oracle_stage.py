@@ -94,3 +94,47 @@ def test_validate_rejects_overlapping_destinations_and_dst_over_live_source():
     # the same plan is fine once the clashing source chunk is dirty (it is then not read)
     bm = np.array([0b10], np.uint8)
     assert orc.stage_validate(buf, buf, buf, [(0, 0, 2048, 512, 0), (2100, 512, 3000, 512, 1)], bm)
+
+
+def test_prestage_writes_unblocked_chunks_and_updates_bitmaps():
+    plan, total, weights, staging, slots = _setup(5, [9000, 4096, 100, 20000], 2048)
+    staging[:] = 0x77
+    n = len(plan)
+    g = wl.rng(402)
+    blocked = g.uniform(size=n) < 0.3
+    staged = np.zeros((n + 7) // 8, np.uint8)
+    dirty = np.packbits(g.uniform(size=n) < 0.5, bitorder="little")
+    dirty0 = np.unpackbits(dirty, bitorder="little")[:n].astype(bool)
+    entries = [(off, off, off, nb, cid) for off, nb, cid in plan]
+    st = orc.prestage(staging, weights, entries, np.packbits(blocked, bitorder="little"), staged, dirty)
+    want = np.full(total, 0x77, np.uint8)
+    for off, nb, cid in plan:
+        if not blocked[cid]:
+            want[off:off + nb] = weights[off:off + nb]
+    assert np.array_equal(staging, want)
+    assert np.array_equal(np.unpackbits(staged, bitorder="little")[:n].astype(bool), ~blocked)
+    assert np.array_equal(np.unpackbits(dirty, bitorder="little")[:n].astype(bool), dirty0 & blocked)
+    assert st.h2d_bytes == sum(nb for _, nb, c in plan if not blocked[c])
+    assert st.missing_chunks == int(blocked.sum()) and st.dirty_chunks == int((dirty0 & ~blocked).sum())
+
+
+def test_mark_dirty_is_interval_overlap_over_staged_chunks():
+    plan, total, weights, staging, slots = _setup(6, [5000, 300, 12000], 1024)
+    n = len(plan)
+    g = wl.rng(403)
+    entries = [(off, off, off, nb, cid) for off, nb, cid in plan]
+    for _ in range(60):
+        staged_b = g.uniform(size=n) < 0.7
+        staged = np.packbits(staged_b, bitorder="little")
+        dirty = np.zeros_like(staged)
+        a = int(g.integers(0, total)); b = int(g.integers(0, 4000))
+        changed = orc.mark_dirty(staging, entries, a, b, staged, dirty)
+        want = np.array([staged_b[c] and b > 0 and off < a + b and a < off + nb for off, nb, c in plan])
+        assert np.array_equal(np.unpackbits(dirty, bitorder="little")[:n].astype(bool), want)
+        assert changed == int(want.sum())
+        assert orc.mark_dirty(staging, entries, a, b, staged, dirty) == 0      # idempotent
+    # a staged chunk next to, but not touching, the allocation stays clean
+    dirty = np.zeros((n + 7) // 8, np.uint8)
+    off, nb, cid = plan[3]
+    assert orc.mark_dirty(staging, entries, off + nb, 10, None, dirty) == (1 if plan[4][0] == off + nb else 0)
+    assert not (dirty[cid >> 3] >> (cid & 7)) & 1
