@@ -307,6 +307,30 @@ talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int
                                const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
                                void *stream);
 
+/* Sec. 4.4 pre-staging, the step that runs while the current model is still serving:
+ * for every plan entry, the authoritative HOST bytes (src_host, pinned) are written to
+ * the chunk's place in the staging region (src_dev, a DEVICE address inside unused KV
+ * rows), unless bit chunk_id of blocked_bitmap is set (those rows currently belong to
+ * a KV allocation, so the chunk stays unstaged).  chunk_id must be >= 0.  For each
+ * chunk written, its bit in staged_bitmap (HOST, in/out, nullable) is set and its
+ * bit in dirty_bitmap (HOST, in/out, nullable) is cleared.  dst_dev is ignored.
+ * stats (nullable): h2d_bytes = bytes written, missing_chunks = chunks skipped,
+ * dirty_chunks = dirty bits cleared, d2d_bytes = 0.  Copy-engine transfers on
+ * `stream`; bitmaps are updated before return, the data lands when the stream gets
+ * there.  Errors: INVALID_ARG, HOST_NOT_PINNED, OVERLAP (two written staging ranges
+ * intersect). */
+talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                  const uint8_t *blocked_bitmap, uint8_t *staged_bitmap,
+                                  uint8_t *dirty_bitmap, talaria_stage_stats_t *stats, void *stream);
+
+/* Sec. 4.4: "marks a chunk dirty if a concurrent prefill allocation takes rows that
+ * overlap the chunk's staging range".  Pure host arithmetic: sets the dirty bit of
+ * every staged chunk (all chunks when staged_bitmap is NULL) whose staging bytes
+ * [src_dev, src_dev+bytes) intersect [alloc_base, alloc_base+alloc_bytes).  Returns the
+ * number of bits that changed from clean to dirty. */
+int64_t talaria_mark_dirty(const talaria_copy_t *plan, int64_t n, const void *alloc_base,
+                           int64_t alloc_bytes, const uint8_t *staged_bitmap, uint8_t *dirty_bitmap);
+
 /* ---- completion, errors, counters ------------------------------------------ */
 
 /* Sec. 4.3 / App. B "Switch barrier": block the host until everything enqueued on

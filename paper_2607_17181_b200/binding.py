@@ -112,6 +112,8 @@ _SIGNATURES = {
     "talaria_kv_offload_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
     "talaria_kv_restore_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
     "talaria_stage": (C.c_int32, [_P, _P, C.c_int64, _P, C.POINTER(StageStats), _P]),
+    "talaria_prestage": (C.c_int32, [_P, _P, C.c_int64, _P, _P, _P, C.POINTER(StageStats), _P]),
+    "talaria_mark_dirty": (C.c_int64, [_P, C.c_int64, _P, C.c_int64, _P, _P]),
     "talaria_sync": (C.c_int32, [_P, _P]),
     "talaria_strerror": (C.c_char_p, [C.c_int32]),
     "talaria_last_cuda_error": (C.c_int32, [_P]),
@@ -317,6 +319,22 @@ class Talaria:
         self._check(lib().talaria_stage(self._h, _ptr(plan), plan.size, _ptr(bm), C.byref(st),
                                         _stream_ptr(stream)), "talaria_stage")
         return st
+
+    def prestage(self, plan: np.ndarray, blocked_bitmap, staged_bitmap: np.ndarray, dirty_bitmap: np.ndarray,
+                 stream=None) -> StageStats:
+        """staged_bitmap / dirty_bitmap: uint8 numpy arrays updated in place."""
+        plan = np.ascontiguousarray(plan, dtype=COPY_DTYPE)
+        bl = None if blocked_bitmap is None else np.ascontiguousarray(blocked_bitmap, dtype=np.uint8)
+        st = StageStats()
+        self._check(lib().talaria_prestage(self._h, _ptr(plan), plan.size, _ptr(bl), _ptr(staged_bitmap),
+                                           _ptr(dirty_bitmap), C.byref(st), _stream_ptr(stream)), "talaria_prestage")
+        return st
+
+    @staticmethod
+    def mark_dirty(plan: np.ndarray, alloc_base: int, alloc_bytes: int, staged_bitmap, dirty_bitmap: np.ndarray) -> int:
+        plan = np.ascontiguousarray(plan, dtype=COPY_DTYPE)
+        return int(lib().talaria_mark_dirty(_ptr(plan), plan.size, alloc_base, alloc_bytes, _ptr(staged_bitmap),
+                                            _ptr(dirty_bitmap)))
 
     # -- completion and counters ---------------------------------------------
     def sync(self, stream=None):

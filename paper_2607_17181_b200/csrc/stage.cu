@@ -234,7 +234,94 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   return TALARIA_OK;
 }
 
+// Pre-staging (Sec. 4.4): authoritative host bytes -> the chunk's place in the staging
+// region, for every chunk whose rows are not blocked by a KV allocation.  Copy-engine
+// H2D, merged over neighbouring chunks, on the caller's stream.
+static talaria_status_t prestage_impl(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                      const uint8_t *blocked, uint8_t *staged, uint8_t *dirty,
+                                      talaria_stage_stats_t *stats, cudaStream_t stream) {
+  if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
+  talaria_stage_stats_t st{0, 0, 0, 0};
+  struct HostRun { const char *h; char *d; int64_t bytes; };
+  std::vector<HostRun> runs;
+  auto bit = [](const uint8_t *bm, int64_t i) { return (bm[i >> 3] >> (i & 7)) & 1; };
+  for (int64_t k = 0; k < n; ++k) {
+    const talaria_copy_t &c = plan[k];
+    if (c.bytes < 0 || c.chunk_id < 0 || !c.src_dev || !c.src_host) return TALARIA_ERR_INVALID_ARG;
+  }
+  if (ctx->cfg.validate) {           // staging ranges that are written must not overlap each other
+    std::vector<Range> dsts;
+    for (int64_t k = 0; k < n; ++k)
+      if (plan[k].bytes > 0 && !(blocked && bit(blocked, plan[k].chunk_id)))
+        dsts.push_back({(uintptr_t)plan[k].src_dev, (uintptr_t)plan[k].src_dev + (uintptr_t)plan[k].bytes});
+    if (any_overlap_sorted(dsts)) return TALARIA_ERR_OVERLAP;
+  }
+  for (int64_t k = 0; k < n; ++k) {
+    const talaria_copy_t &c = plan[k];
+    if (blocked && bit(blocked, c.chunk_id)) continue;
+    if (c.bytes == 0) continue;
+    const char *h = (const char *)c.src_host;
+    char *d = (char *)c.src_dev;
+    if (!runs.empty() && runs.back().h + runs.back().bytes == h && runs.back().d + runs.back().bytes == d) {
+      runs.back().bytes += c.bytes;
+    } else {
+      void *alias;
+      TAL_TRY(mapped_pointer(ctx, h, &alias));
+      runs.push_back(HostRun{h, d, c.bytes});
+    }
+  }
+  for (const HostRun &r : runs) {
+    TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, stream));
+    ctx->counters.memcpy_calls++;
+  }
+  // bookkeeping only after every copy was accepted
+  for (int64_t k = 0; k < n; ++k) {
+    const talaria_copy_t &c = plan[k];
+    if (blocked && bit(blocked, c.chunk_id)) { st.missing_chunks++; continue; }
+    st.h2d_bytes += c.bytes;
+    if (staged) staged[c.chunk_id >> 3] |= (uint8_t)(1u << (c.chunk_id & 7));
+    if (dirty && bit(dirty, c.chunk_id)) {
+      dirty[c.chunk_id >> 3] &= (uint8_t)~(1u << (c.chunk_id & 7));
+      st.dirty_chunks++;
+    }
+  }
+  ctx->counters.payload_bytes += st.h2d_bytes;
+  if (stats) *stats = st;
+  return TALARIA_OK;
+}
+
 }  // namespace tal
+
+extern "C" talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                             const uint8_t *blocked_bitmap, uint8_t *staged_bitmap,
+                                             uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
+                                             void *stream) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  tal::DeviceGuard g(ctx->device);
+  if (!g.ok) return TALARIA_ERR_CUDA;
+  return tal::prestage_impl(ctx, plan, n, blocked_bitmap, staged_bitmap, dirty_bitmap, stats, (cudaStream_t)stream);
+}
+
+extern "C" int64_t talaria_mark_dirty(const talaria_copy_t *plan, int64_t n, const void *alloc_base,
+                                      int64_t alloc_bytes, const uint8_t *staged_bitmap,
+                                      uint8_t *dirty_bitmap) {
+  if (!plan || n <= 0 || !dirty_bitmap || alloc_bytes <= 0) return 0;
+  const uintptr_t a0 = (uintptr_t)alloc_base, a1 = a0 + (uintptr_t)alloc_bytes;
+  int64_t changed = 0;
+  for (int64_t k = 0; k < n; ++k) {
+    const talaria_copy_t &c = plan[k];
+    if (c.bytes <= 0 || c.chunk_id < 0 || !c.src_dev) continue;
+    const int64_t id = c.chunk_id;
+    if (staged_bitmap && !((staged_bitmap[id >> 3] >> (id & 7)) & 1)) continue;
+    const uintptr_t s0 = (uintptr_t)c.src_dev, s1 = s0 + (uintptr_t)c.bytes;
+    if (s0 < a1 && a0 < s1 && !((dirty_bitmap[id >> 3] >> (id & 7)) & 1)) {
+      dirty_bitmap[id >> 3] |= (uint8_t)(1u << (id & 7));
+      ++changed;
+    }
+  }
+  return changed;
+}
 
 extern "C" talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
                                           const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,

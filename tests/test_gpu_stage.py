@@ -114,3 +114,76 @@ def test_plan_errors(ctx):
     assert status(arr) == tb.ERR_HOST_NOT_PINNED
     arr[1] = (a.ptr, 0, 0, 512, 1, 0)
     assert status(arr) == tb.ERR_INVALID_ARG
+
+
+def test_prestage_then_dirty_marking_then_switch(ctx):
+    """The whole Sec. 4.4 protocol: pre-stage what is not blocked, a KV allocation scribbles over
+    part of the staging region and marks those chunks dirty, the switch then takes clean chunks
+    D2D and dirty / unstaged ones from host; every slot must end up with the authoritative bytes."""
+    sizes = [300_000, 70_001, 5, 1 << 20, 33_333, 4096 * 192 * 2]
+    plan, total = wl.stage_plan(sizes, 64 << 10)
+    g = wl.rng(601)
+    n = len(plan)
+    weights = g.integers(0, 256, size=total, dtype=np.uint8)
+    host = GuardedPinned(total); host.np[:] = weights
+    staging = GuardedDevice(total, np.full(total, 0x77, np.uint8))
+    slots = GuardedDevice(total, np.full(total, 0xEE, np.uint8))
+    arr = np.zeros(n, tb.COPY_DTYPE)
+    for k, (off, nb, cid) in enumerate(plan):
+        arr[k] = (staging.ptr + off, host.ptr + off, slots.ptr + off, nb, cid, 0)
+    blocked = g.uniform(size=n) < 0.25
+    staged, dirty = np.zeros((n + 7) // 8, np.uint8), np.zeros((n + 7) // 8, np.uint8)
+    st = ctx.prestage(arr, np.packbits(blocked, bitorder="little"), staged, dirty)
+    ctx.sync()
+    # oracle mirror
+    o_staging = np.full(total, 0x77, np.uint8)
+    o_staged, o_dirty = np.zeros_like(staged), np.zeros_like(dirty)
+    entries = [(off, off, off, nb, cid) for off, nb, cid in plan]
+    ost = orc.prestage(o_staging, weights, entries, np.packbits(blocked, bitorder="little"), o_staged, o_dirty)
+    assert np.array_equal(staging.read(), o_staging) and np.array_equal(staged, o_staged)
+    assert (st.h2d_bytes, st.missing_chunks, st.dirty_chunks) == (ost.h2d_bytes, ost.missing_chunks, ost.dirty_chunks)
+    # a prefill allocation takes rows in the middle of the staging region
+    a_off, a_len = total // 3, 200_000
+    junk = g.integers(0, 256, size=a_len, dtype=np.uint8)
+    view = staging.read(); view[a_off:a_off + a_len] = junk; staging.write(view)
+    o_staging[a_off:a_off + a_len] = junk
+    changed = tb.Talaria.mark_dirty(arr, staging.ptr + a_off, a_len, staged, dirty)
+    assert changed == orc.mark_dirty(o_staging, entries, a_off, a_len, o_staged, o_dirty) > 0
+    assert np.array_equal(dirty, o_dirty)
+    # switch: unstaged chunks are "missing"
+    is_staged = np.unpackbits(staged, bitorder="little")[:n].astype(bool)
+    sw = arr.copy()
+    sw["src_dev"][~is_staged] = 0
+    sst = ctx.stage(sw, dirty)
+    ctx.sync()
+    covered = np.zeros(total, bool)                      # alignment gaps between tensors are never copied
+    for off, nb, _ in plan:
+        covered[off:off + nb] = True
+    assert np.array_equal(slots.read(), np.where(covered, weights, 0xEE))
+    assert sst.missing_chunks == int((~is_staged).sum()) and sst.dirty_chunks == changed
+    # staging again clears the dirty bits of rewritten chunks
+    st2 = ctx.prestage(arr, None, staged, dirty)
+    ctx.sync()
+    assert st2.dirty_chunks == changed and not dirty.any()
+    assert np.array_equal(staging.read()[covered], weights[covered])
+    assert slots.guards_ok() and staging.guards_ok() and host.guards_ok()
+
+
+def test_prestage_errors(ctx):
+    a = GuardedDevice(8192, np.zeros(8192, np.uint8))
+    host = GuardedPinned(8192)
+    arr = np.zeros(2, tb.COPY_DTYPE)
+    arr[0] = (a.ptr, host.ptr, 0, 1024, 0, 0)
+    arr[1] = (a.ptr + 512, host.ptr + 2048, 0, 1024, 1, 0)
+    bm = np.zeros(1, np.uint8)
+    with pytest.raises(tb.TalariaError) as e:
+        ctx.prestage(arr, None, bm, bm.copy())
+    assert e.value.status == tb.ERR_OVERLAP and not bm.any()
+    arr[1] = (a.ptr + 2048, np.zeros(1024, np.uint8).ctypes.data, 0, 1024, 1, 0)
+    with pytest.raises(tb.TalariaError) as e:
+        ctx.prestage(arr, None, bm, bm.copy())
+    assert e.value.status == tb.ERR_HOST_NOT_PINNED and not bm.any()
+    arr[1] = (a.ptr + 2048, host.ptr + 2048, 0, 1024, -1, 0)
+    with pytest.raises(tb.TalariaError) as e:
+        ctx.prestage(arr, None, bm, bm.copy())
+    assert e.value.status == tb.ERR_INVALID_ARG
