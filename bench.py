@@ -191,6 +191,37 @@ def link_ceiling(torch, dev, nbytes=1 << 30, reps=6):
     return best
 
 
+def run_other_workload(args):
+    """configs[2..4]: measurement lines of their own (the default line is configs[1])."""
+    import torch
+    from paper_2607_17181_b200 import bench_configs as bc
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ceilings = link_ceiling(torch, dev)
+    peaks, kind = measured_peaks()
+    sampler = ClockSampler(local)
+    sampler.start()
+    if args.workload == "long":
+        res = bc.run_long(torch, dev, ceilings)
+        unit = "GB/s restore into isolated blocks (mean over cases)"
+    elif args.workload == "stage":
+        res = bc.run_stage(torch, dev, ceilings, float(peaks["hbm_gbs"]))
+        unit = "GB/s read+write of the D2D staging kernel, all chunks clean, alone"
+    else:
+        res = bc.run_replay(torch, dev, ceilings)
+        unit = "GB/s aggregate offload+restore payload over the drained transfer calls"
+    clocks = sampler.stop()
+    line = {"metric": METRIC, "value": res.pop("value"), "unit": unit, "n_gpus": 1, "higher_is_better": True,
+            "dtype": "u8", "data": "synthetic", "vs_baseline": None, "config": {"workload": res.pop("workload")},
+            "ceilings": {"h2d_gbs": ceilings["h2d"], "d2h_gbs": ceilings["d2h"], "hbm_gbs": peaks["hbm_gbs"],
+                         "hbm_kind": kind, "nominal_pcie5_x16_gbs": PCIE5_X16_GBS}, "clocks": clocks}
+    line.update(res)
+    print(json.dumps(line))
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -447,6 +478,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 zero-copy, 2 bounce+DMA, 3 per-run DMA")
     ap.add_argument("--scale", default="full", choices=["full", "small"], help="small = profiling-sized workload")
+    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay"],
+                    help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -454,6 +487,8 @@ def main():
     apply_scale(args.scale)
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "session":
+        run_other_workload(args)
     else:
         run_gpu(args)
 

@@ -1,0 +1,239 @@
+"""Measurements of the other benchmark configurations (`bench.py --workload ...`).
+
+`bench.py`'s default line is the one-session workload; these are the long-context,
+staging-plus-restore and session-replay workloads.  Each function returns one dict
+(printed as a JSON line by bench.py).  All timing is CUDA events on the launching
+streams; parity for the same workloads lives in the tests.
+"""
+from __future__ import annotations
+
+import statistics
+import time
+from typing import Dict, List
+
+import numpy as np
+
+from . import binding as tb
+from . import workloads as wl
+from .replay import ReplayDriver
+
+PCIE5_X16_GBS = 63.0
+
+
+def _pool(torch, dev, shape, num_blocks, seed):
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    planes = []
+    for _ in range(shape.num_layers * shape.num_planes):
+        t = torch.empty(num_blocks * shape.chunk_bytes // 2, dtype=torch.bfloat16, device=dev)
+        t.normal_(generator=gen)
+        planes.append(t)
+    kv, keep = tb.kv_layout(shape, [t.data_ptr() for t in planes], num_blocks)
+    return planes, kv, keep
+
+
+def _timed(torch, stream, fn, reps):
+    fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return statistics.median(ts)
+
+
+def run_long(torch, dev, ceilings, reps=3) -> Dict:
+    """Long-context session (105,000 tokens) at 16- and 32-token blocks: offload, restore into
+    isolated single free blocks, and the same restore while a second session (25,000 tokens) is
+    offloaded on another stream."""
+    out = {"workload": "configs[2]: 105,000-token session, Qwen3-235B KV shape, restore into isolated free "
+                       "blocks, second-session offload overlapped", "cases": []}
+    pinned = torch.empty(20_218_380_288, dtype=torch.uint8, pin_memory=True)
+    for B, order in ((16, "PF"), (32, "PF"), (16, "LF")):
+        shape = wl.QWEN235 if B == 16 else wl.QWEN235_B32
+        NB = 16_384 if B == 16 else 8_192
+        torch.cuda.empty_cache()
+        planes, kv, keep = _pool(torch, dev, shape, NB, 30 + B)
+        g = wl.rng(3, B)
+        n, n2 = shape.blocks_for(105_000), shape.blocks_for(25_000)
+        even = np.arange(0, NB, 2, dtype=np.int32)
+        src = np.ascontiguousarray(g.permutation(even)[:n])
+        second = np.ascontiguousarray(g.permutation(np.setdiff1d(even, src))[:n2])
+        dst = wl.isolated_table(g, NB, n)
+        size = n * shape.bytes_per_block
+        image = pinned[:size]
+        hl = tb.host_layout(wl.dense_strides(shape, n, order), size)
+        image2 = torch.empty(n2 * shape.bytes_per_block, dtype=torch.uint8, pin_memory=True)
+        hl2 = tb.host_layout(wl.dense_strides(shape, n2, "PF"), image2.numel())
+        ctx = tb.Talaria(dev.index or 0)
+        sa, sb = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        t_off = _timed(torch, sa, lambda: ctx.kv_offload(kv, src, 0, n, image, hl, stream=sa), reps)
+        t_res = _timed(torch, sa, lambda: ctx.kv_restore(kv, dst, 0, n, image, hl, stream=sa), reps)
+        both = []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            e[0].record(sa); e[2].record(sb)
+            ctx.kv_restore(kv, dst, 0, n, image, hl, stream=sa); e[1].record(sa)
+            ctx.kv_offload(kv, second, 0, n2, image2, hl2, stream=sb); e[3].record(sb)
+            torch.cuda.synchronize()
+            both.append((e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3])))
+        t_r2, t_o2 = min(both)
+        toks = wl.tokens(g, 105_000)
+        cont = wl.continuation(g, toks, 110_000, 100_000)
+        d_s, d_c = torch.from_numpy(toks).to(dev), torch.from_numpy(cont).to(dev)
+        d_h = torch.empty(110_000 // B, dtype=torch.int64, device=dev)
+        d_r = torch.zeros(4, dtype=torch.int64, device=dev)
+        t_m = _timed(torch, sa, lambda: [ctx.prefix_match(1, d_c, [0, 110_000], d_s, [0, 105_000], None, B,
+                                                          wl.HASH_SEED, d_h, d_r, stream=sa) for _ in range(50)], reps) / 50
+        out["cases"].append({
+            "block_tokens": B, "host_layout": order, "blocks": n, "payload_bytes": size,
+            "offload_gbs": size / t_off / 1e6, "offload_frac_of_d2h_ceiling": size / t_off / 1e6 / ceilings["d2h"],
+            "restore_isolated_gbs": size / t_res / 1e6, "restore_frac_of_h2d_ceiling": size / t_res / 1e6 / ceilings["h2d"],
+            "overlapped": {"restore_gbs": size / t_r2 / 1e6, "second_offload_gbs": image2.numel() / t_o2 / 1e6},
+            "prefix_match_us": t_m * 1e3, "variant": int(ctx.get_counters().last_variant)})
+        ctx.destroy()
+        del planes, image2
+    out["value"] = statistics.mean(c["restore_isolated_gbs"] for c in out["cases"])
+    return out
+
+
+def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
+    """D2D weight staging (58.96 GB in 2 MiB chunks) with a 25,000-token KV restore on a second
+    stream, at 0 %, 1 % and 36 % dirty chunks."""
+    ws = wl.moe_weight_set()
+    plan, span = wl.stage_plan(ws.sizes, 2 << 20)
+    total = sum(nb for _, nb, _ in plan)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(55)
+    staging = torch.empty(span, dtype=torch.uint8, device=dev)
+    for off in range(0, span, 1 << 30):
+        m = min(1 << 30, span - off)
+        staging[off:off + m].view(torch.int16).random_(generator=gen)
+    slots = torch.zeros(span, dtype=torch.uint8, device=dev)
+    shape, NB = wl.QWEN235, 2048
+    nblk = shape.blocks_for(25_000)
+    planes, kv, keep = _pool(torch, dev, shape, NB, 56)
+    g = wl.rng(5)
+    table = np.ascontiguousarray(g.permutation(NB)[:nblk].astype(np.int32))
+    image = torch.empty(nblk * shape.bytes_per_block, dtype=torch.uint8, pin_memory=True)
+    hl = tb.host_layout(wl.dense_strides(shape, nblk, "PF"), image.numel())
+    ctx = tb.Talaria(dev.index or 0)
+    sa, sb = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    out = {"workload": "configs[4]: 58.96 GB weight set staged D2D into stable slots (2 MiB chunks) while a "
+                       "25,000-token KV restore runs on a second stream", "cases": []}
+    n = len(plan)
+    for frac in (0.0, 0.01, 0.36):
+        dirty = g.uniform(size=n) < frac
+        idx = np.nonzero(dirty)[0]
+        host_off = np.zeros(n, np.int64)
+        at = 0
+        for k in idx:
+            host_off[k] = at
+            at += -(-plan[k][1] // 256) * 256
+        host = torch.empty(max(at, 256), dtype=torch.uint8, pin_memory=True)
+        arr = np.zeros(n, tb.COPY_DTYPE)
+        for k, (off, nb, cid) in enumerate(plan):
+            arr[k] = (staging.data_ptr() + off, host.data_ptr() + int(host_off[k]) if dirty[k] else 0,
+                      slots.data_ptr() + off, nb, cid, 0)
+        bitmap = np.packbits(dirty, bitorder="little")
+        h2d = int(sum(plan[k][1] for k in idx))
+        t_alone = _timed(torch, sa, lambda: ctx.stage(arr, bitmap, stream=sa), reps)
+        t_res_alone = _timed(torch, sb, lambda: ctx.kv_restore(kv, table, 0, nblk, image, hl, stream=sb), reps)
+        both = []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            e[0].record(sa); e[2].record(sb)
+            ctx.stage(arr, bitmap, stream=sa); e[1].record(sa)
+            ctx.kv_restore(kv, table, 0, nblk, image, hl, stream=sb); e[3].record(sb)
+            torch.cuda.synchronize()
+            both.append((e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3])))
+        t_st, t_rs = min(both)
+        d2d = total - h2d
+        out["cases"].append({
+            "dirty_fraction": frac, "d2d_bytes": d2d, "h2d_bytes": h2d,
+            "stage_alone_ms": t_alone, "stage_with_restore_ms": t_st,
+            "d2d_gbs_read_write_alone": (2 * d2d / t_alone / 1e6) if frac == 0 else None,
+            "frac_of_hbm_peak_alone": (2 * d2d / t_alone / 1e6 / hbm_peak) if frac == 0 else None,
+            "h2d_gbs_alone": (h2d / t_alone / 1e6) if h2d else None,
+            "restore_alone_gbs": image.numel() / t_res_alone / 1e6,
+            "restore_with_stage_gbs": image.numel() / t_rs / 1e6})
+        del host
+    ctx.destroy()
+    out["value"] = out["cases"][0]["d2d_gbs_read_write_alone"]
+    return out
+
+
+def run_replay(torch, dev, ceilings, max_calls=160, host_budget_gb=60.0) -> Dict:
+    """Session-replay mix at the full KV shape: 30 sessions, pool capped at 60 GB (19,479
+    blocks), whole-session LRU eviction to pinned host images, restore on return."""
+    shape = wl.QWEN235
+    pool_blocks = int(60e9) // shape.bytes_per_block
+    torch.cuda.empty_cache()
+    planes, kv, keep = _pool(torch, dev, shape, pool_blocks, 44)
+    ctx = tb.Talaria(dev.index or 0)
+    # one pinned arena, handed out in order and recycled when full (images are dropped on restore)
+    arena = torch.empty(int(host_budget_gb * 1.25e9), dtype=torch.uint8, pin_memory=True)
+    cursor = [0]
+
+    def alloc_pinned(nbytes):
+        nbytes_al = -(-nbytes // 4096) * 4096
+        if cursor[0] + nbytes_al > arena.numel():
+            cursor[0] = 0
+        t = arena[cursor[0]:cursor[0] + nbytes]
+        cursor[0] += nbytes_al
+        return t
+
+    scratch = torch.empty(131_072 // 16 * shape.bytes_per_block, dtype=torch.uint8, device=dev)
+
+    def content(sid, k, nbytes):                 # synthetic "prefill output", generated on the device
+        v = scratch[:nbytes]
+        v.view(torch.int64).random_()
+        return v
+
+    drv = ReplayDriver(ctx, shape, kv, pool_blocks, int(host_budget_gb * 1e9), wl.HASH_SEED, content, alloc_pinned,
+                       lambda a: a, order="PF")
+    schedule = wl.session_replay()[:max_calls]
+    streams, tg = {}, wl.rng(4, 2)
+    groups, cur = [], []
+    for c in schedule:
+        if len(cur) == 4 or any(x.session == c.session for x in cur):
+            groups.append(cur)
+            cur = []
+        cur.append(c)
+    if cur:
+        groups.append(cur)
+    match_us: List[float] = []
+    t0 = time.perf_counter()
+    for grp in groups:
+        calls = []
+        for c in grp:
+            prev = streams.get(c.session)
+            toks = wl.tokens(tg, c.prompt_tokens) if prev is None else \
+                wl.continuation(tg, prev, c.prompt_tokens, min(c.shared_tokens, prev.size))
+            calls.append((c.session, c.index, toks))
+            streams[c.session] = toks
+        drv.run_group(calls)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    st = drv.stats
+    ctx.destroy()
+    return {"workload": f"configs[3]: session-replay mix, first {len(schedule)} calls of 30 sessions, 60 GB pool "
+                        f"({pool_blocks} blocks), LRU eviction, host budget {host_budget_gb:.0f} GB",
+            "calls": st.calls, "device_hits": st.device_hits, "host_restores": st.host_restores,
+            "recomputes": st.recomputes, "capacity_misses": st.capacity_misses, "evictions": st.evictions,
+            "offload_bytes": st.offload_bytes, "restore_bytes": st.restore_bytes,
+            "prompt_tokens": st.prompt_tokens, "reused_tokens": st.reused_tokens,
+            "reused_fraction": st.reused_tokens / max(st.prompt_tokens, 1),
+            "offload_gbs": st.offload_bytes / max(st.offload_s, 1e-9) / 1e9,
+            "restore_gbs": st.restore_bytes / max(st.restore_s, 1e-9) / 1e9,
+            "batched_match_us_per_group_e2e_from_host": st.match_s / max(st.match_calls, 1) * 1e6,
+            "tokens_per_s_of_prefix_preserved": st.reused_tokens / max(wall, 1e-9),
+            "timing": "host wall clock around each drained batched call (transfers are 0.1 s and longer)",
+            "wall_s_including_host_side_generation": wall,
+            "value": (st.offload_bytes + st.restore_bytes) / max(st.offload_s + st.restore_s, 1e-9) / 1e9}

@@ -103,8 +103,15 @@ struct Range {
   uintptr_t lo, hi;
 };
 
+static void sort_ranges(std::vector<Range> &a) {
+  // plans are normally written in address order: skip the sort when they already are
+  bool sorted = true;
+  for (size_t k = 1; k < a.size() && sorted; ++k) sorted = a[k - 1].lo <= a[k].lo;
+  if (!sorted) std::sort(a.begin(), a.end(), [](const Range &x, const Range &y) { return x.lo < y.lo; });
+}
+
 static bool any_overlap_sorted(std::vector<Range> &a) {
-  std::sort(a.begin(), a.end(), [](const Range &x, const Range &y) { return x.lo < y.lo; });
+  sort_ranges(a);
   for (size_t k = 1; k < a.size(); ++k)
     if (a[k].lo < a[k - 1].hi) return true;
   return false;
@@ -112,7 +119,7 @@ static bool any_overlap_sorted(std::vector<Range> &a) {
 
 // a sorted & disjoint; does any range of b intersect a range of a?
 static bool cross_overlap(const std::vector<Range> &a, std::vector<Range> &b) {
-  std::sort(b.begin(), b.end(), [](const Range &x, const Range &y) { return x.lo < y.lo; });
+  sort_ranges(b);
   size_t i = 0;
   for (const Range &r : b) {
     while (i < a.size() && a[i].hi <= r.lo) ++i;
@@ -163,9 +170,8 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
     if (cross_overlap(dsts, srcs)) return TALARIA_ERR_OVERLAP;
   }
 
-  // ---- H2D leg: merged copy-engine copies on an internal stream ----------
-  // Every host source is checked before anything is enqueued, so a rejected plan
-  // leaves no partial copy behind.
+  // ---- H2D leg, part 1: merge neighbouring host-sourced chunks and check every host
+  // source before anything is enqueued, so a rejected plan leaves no partial copy behind.
   struct HostRun { const char *h; char *d; int64_t bytes; };
   std::vector<HostRun> runs;
   for (int64_t k = 0; k < n;) {
@@ -182,17 +188,14 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
     runs.push_back(r);
     k = j;
   }
+  // The internal stream forks from the caller's stream BEFORE the D2D kernel is launched, so
+  // the host-sourced copies depend only on earlier work and run next to the kernel.
   BounceLane &ln = ctx->lane[1];
   const bool forked = !runs.empty();
   if (forked) {
     TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
     TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
-    for (const HostRun &r : runs) {
-      TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
-      ctx->counters.memcpy_calls++;
-    }
   }
-
   // ---- D2D leg ---------------------------------------------------------------
   if (n_clean > 0 && st.d2d_bytes > 0) {
     // count tiles first so the descriptor (entries, then one int32 per span) can be sized
@@ -225,7 +228,12 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
     ctx->counters.kernel_launches++;
     TAL_TRY(release_slot(ctx, slot, stream));
   }
+  // ---- H2D leg, part 2: enqueued second, so the kernel is already running meanwhile
   if (forked) {
+    for (const HostRun &r : runs) {
+      TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
+      ctx->counters.memcpy_calls++;
+    }
     TAL_CUDA(ctx, cudaEventRecord(ln.done[0], ln.s[0]));
     TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[0], 0));
   }

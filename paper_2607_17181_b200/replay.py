@@ -23,6 +23,7 @@ the CPU oracle; this module itself never imports the oracle.
 from __future__ import annotations
 
 import heapq
+import time
 from dataclasses import dataclass, field
 from typing import Callable, Dict, List, Optional, Sequence, Tuple
 
@@ -56,6 +57,10 @@ class ReplayStats:
     restore_bytes: int = 0
     reused_tokens: int = 0
     prompt_tokens: int = 0
+    offload_s: float = 0.0        # host wall time of the batched calls, drained
+    restore_s: float = 0.0
+    match_s: float = 0.0
+    match_calls: int = 0
 
 
 class ReplayDriver:
@@ -119,8 +124,10 @@ class ReplayDriver:
         if freed < need:
             raise RuntimeError("pool too small for this call even after evicting every other session")
         if xfers:
+            t0 = time.perf_counter()
             self.ctx.kv_offload_batch(self.kv, xfers)
             self.ctx.sync()                                   # drain before the blocks are reused (App. B)
+            self.stats.offload_s += time.perf_counter() - t0
             self.stats.offload_bytes += sum(x[2] for x in xfers) * self.shape.bytes_per_block
         for s in chosen:
             kept = s.image is not None
@@ -149,7 +156,10 @@ class ReplayDriver:
         stored = stored if stored.size else np.zeros(1, np.uint64)
         out_h = np.zeros(max(int(sum(c.size // B for c in conts)), 1), np.uint64)
         res = np.zeros(len(calls), tb.MATCH_DTYPE)
+        t0 = time.perf_counter()
         self.ctx.prefix_match_host(len(calls), cont_all, co, sess_all, so, stored, B, self.seed, out_h, res)
+        self.stats.match_s += time.perf_counter() - t0
+        self.stats.match_calls += 1
         self.log.append(("match", [(sid, k) for sid, k, _ in calls], res.copy(), out_h.copy()))
         # ---- residency decisions, allocation ----------------------------------
         restores, plans, at = [], [], 0
@@ -190,8 +200,10 @@ class ReplayDriver:
             self.stats.reused_tokens += reuse * B
         # ---- restore the matched prefixes of all returning sessions in one call ----
         if restores:
+            t0 = time.perf_counter()
             self.ctx.kv_restore_batch(self.kv, [r[:5] for r in restores])
             self.ctx.sync()
+            self.stats.restore_s += time.perf_counter() - t0
             self.stats.restore_bytes += sum(r[2] for r in restores) * self.shape.bytes_per_block
             for table, _, reuse, _, _, sid, n_img in restores:
                 self.log.append(("restore", sid, table[:reuse].copy(), n_img))
@@ -203,7 +215,7 @@ class ReplayDriver:
             if m:
                 img = self.content(s.sid, k, m * self.shape.bytes_per_block)
                 d_img = self.to_device(img)
-                il = tb.host_layout(wl.dense_strides(self.shape, m, "PF"), img.size)
+                il = tb.host_layout(wl.dense_strides(self.shape, m, "PF"), m * self.shape.bytes_per_block)
                 self.ctx.kv_scatter(self.kv, table, reuse, m, d_img, il)
                 self.ctx.sync()
                 self.log.append(("fill", s.sid, k, table[reuse:].copy()))
