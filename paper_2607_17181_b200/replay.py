@@ -61,6 +61,7 @@ class ReplayStats:
     restore_s: float = 0.0
     match_s: float = 0.0
     match_calls: int = 0
+    match_times: List[float] = field(default_factory=list)
 
 
 class ReplayDriver:
@@ -159,6 +160,7 @@ class ReplayDriver:
         t0 = time.perf_counter()
         self.ctx.prefix_match_host(len(calls), cont_all, co, sess_all, so, stored, B, self.seed, out_h, res)
         self.stats.match_s += time.perf_counter() - t0
+        self.stats.match_times.append(time.perf_counter() - t0)
         self.stats.match_calls += 1
         self.log.append(("match", [(sid, k) for sid, k, _ in calls], res.copy(), out_h.copy()))
         # ---- residency decisions, allocation ----------------------------------
