@@ -90,6 +90,9 @@ def lib():
             f.restype = C.c_int32
             f.argtypes = [C.POINTER(_KvLayout), C.c_void_p, C.c_int64, C.c_int64, C.c_void_p,
                           C.POINTER(_HostLayout)]
+        _lib.orc_kv_pages.restype = C.c_int32
+        _lib.orc_kv_pages.argtypes = [C.POINTER(_KvLayout), C.c_void_p, C.c_int64, C.c_int64, C.c_void_p,
+                                      C.c_int64, C.c_void_p, C.c_int32]
         _lib.orc_stage.restype = C.c_int32
         _lib.orc_stage.argtypes = [C.POINTER(_Copy), C.c_int64, C.c_void_p, C.POINTER(_StageStats)]
         _lib.orc_prestage.restype = C.c_int32
@@ -242,6 +245,21 @@ def kv_offload(shape, planes, block_table, first, n, host, strides, form="chunk"
 def kv_restore(shape, planes, block_table, first, n, host, strides, form="chunk"):
     """pool_{l,p}[bt[first+i]] <- host[l,p,i] for i<n (planes are written)."""
     _kv_call(f"orc_kv_restore_{form}", shape, planes, block_table, first, n, host, strides)
+
+
+def kv_pages(shape, planes, block_table, first, n, host_pool: np.ndarray, page_offsets, to_host: bool):
+    """One page-first slab per logical block at host_pool[page_offsets[i]:]: offload when
+    to_host, else restore (planes are written)."""
+    bt = _i32(block_table)
+    po = np.ascontiguousarray(page_offsets, dtype=np.int64)
+    assert po.size >= n and 0 <= first and first + n <= bt.size
+    assert host_pool.dtype == np.uint8 and host_pool.flags.c_contiguous
+    kv, _hl, keep = _kv_args(shape, planes, (0, 0, 0), host_pool)
+    rc = lib().orc_kv_pages(C.byref(kv), _ptr(bt), first, n, host_pool.ctypes.data, host_pool.size, _ptr(po),
+                            1 if to_host else 0)
+    del keep
+    if rc != 0:
+        raise ValueError(f"orc_kv_pages: rc={rc}")
 
 
 # ------------------------------------------------------------------ stage

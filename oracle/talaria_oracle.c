@@ -20,6 +20,10 @@
  *                                   numpy slice cross-check, corrupted-dirty
  *                                   staging test)
  *   orc_prefix_agree      pinned   (App. B "Prefix agreement": brute force)
+ *   orc_kv_offload_pages /
+ *   orc_kv_restore_pages  pinned   (App. C page-first: one slab per logical page; reduces
+ *                                   to the dense page-first image when pages are
+ *                                   consecutive, numpy check for shuffled pages)
  *   orc_prestage /
  *   orc_mark_dirty        pinned   (Sec. 4.4 pre-staging protocol: numpy slice and
  *                                   interval brute force)
@@ -268,6 +272,30 @@ int32_t orc_kv_restore_chunk(const orc_kv_layout_t *kv, const int32_t *bt, int64
                        (size_t)C);
             }
         }
+    return 0;
+}
+
+/* Page-first registry slabs (App. C: "grouped by logical prefix page, with the
+ * per-layer fragments for that page stored under one page descriptor"): logical block
+ * i lives in one slab of layers*planes*C bytes at byte offset page_off[i] of the host
+ * pool, fragments ordered [layer][plane].  to_host: slab <- pool chunk; else pool <- slab. */
+int32_t orc_kv_pages(const orc_kv_layout_t *kv, const int32_t *bt, int64_t first, int64_t n,
+                     uint8_t *host_pool, int64_t pool_bytes, const int64_t *page_off, int32_t to_host)
+{
+    const int64_t C = orc_chunk_bytes(kv);
+    const int64_t slab = (int64_t)kv->num_layers * kv->num_planes * C;
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t b = bt[first + i];
+        if (b < 0 || b >= kv->num_blocks) return -2;
+        if (page_off[i] < 0 || page_off[i] + slab > pool_bytes) return -5;
+        for (int32_t l = 0; l < kv->num_layers; ++l)
+            for (int32_t p = 0; p < kv->num_planes; ++p) {
+                uint8_t *plane = kv->plane_base[l * kv->num_planes + p];
+                uint8_t *frag = host_pool + page_off[i] + ((int64_t)l * kv->num_planes + p) * C;
+                if (to_host) memcpy(frag, plane + b * C, (size_t)C);
+                else         memcpy(plane + b * C, frag, (size_t)C);
+            }
+    }
     return 0;
 }
 

@@ -151,3 +151,36 @@ def test_bad_block_id_is_rejected_and_zero_blocks_is_a_no_op():
     img = np.zeros(2 * shape.bytes_per_block, np.uint8)
     orc.kv_offload(_oshape(shape), planes, np.array([], np.int32), 0, 0, img, wl.dense_strides(shape, 0, "PF"))
     assert not img.any()
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_page_slabs_reduce_to_dense_page_first_and_follow_any_page_order(shape):
+    nb, n = 29, 11
+    planes = _pool(7, shape, nb)
+    g = wl.rng(306)
+    bt = wl.disjoint_tables(g, nb, [n])[0]
+    slab = shape.bytes_per_block
+    dense = np.zeros(n * slab, np.uint8)
+    orc.kv_offload(_oshape(shape), planes, bt, 0, n, dense, wl.dense_strides(shape, n, "PF"))
+    # consecutive pages = the dense page-first image
+    pool = np.full(n * slab, 0x42, np.uint8)
+    orc.kv_pages(_oshape(shape), planes, bt, 0, n, pool, np.arange(n) * slab, True)
+    assert np.array_equal(pool, dense)
+    # shuffled pages with gaps: page i sits where its offset says, everything else untouched
+    order = g.permutation(2 * n)[:n]
+    offs = order.astype(np.int64) * (slab + 16) + 8
+    big = np.full(2 * n * (slab + 16) + 64, 0x42, np.uint8)
+    orc.kv_pages(_oshape(shape), planes, bt, 0, n, big, offs, True)
+    touched = np.zeros(big.size, bool)
+    for i in range(n):
+        assert np.array_equal(big[offs[i]:offs[i] + slab], dense[i * slab:(i + 1) * slab])
+        touched[offs[i]:offs[i] + slab] = True
+    assert np.all(big[~touched] == 0x42)
+    # restore from the shuffled slabs into new blocks equals restore from the dense image
+    bt2 = wl.disjoint_tables(g, nb, [n], exclude=bt)[0]
+    a, b = [p.copy() for p in planes], [p.copy() for p in planes]
+    orc.kv_pages(_oshape(shape), a, bt2, 0, n, big, offs, False)
+    orc.kv_restore(_oshape(shape), b, bt2, 0, n, dense, wl.dense_strides(shape, n, "PF"))
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))
+    with pytest.raises(ValueError):
+        orc.kv_pages(_oshape(shape), planes, bt, 0, n, big, offs + big.size, True)
