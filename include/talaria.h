@@ -268,6 +268,25 @@ talaria_status_t talaria_kv_restore_layered(talaria_ctx *ctx, const talaria_kv_l
                                             const talaria_host_layout_t *hl,
                                             void *const *layer_events, void *stream);
 
+/* Page-first registry slabs (App. C: the host representation "grouped by logical prefix
+ * page, with the per-layer fragments for that page stored under one page descriptor";
+ * Sec. 4.3: slabs of one unified pinned pool).  Logical block i is ONE slab of
+ * num_layers*num_planes*C bytes, fragments ordered [layer][plane], at byte offset
+ * page_offsets[i] (HOST int64[n_blocks]) of the pinned HOST pool (host_pool, pool_bytes).
+ * Slabs may sit anywhere in the pool, in any order: the registry commits, invalidates
+ * and restores at page granularity.
+ *   offload_pages: slab_i <- pool_{l,p}[block_table[first_block+i]]   (slabs must not overlap: OVERLAP)
+ *   restore_pages: pool_{l,p}[new_block_table[first_block+i]] <- slab_i  (DUP_BLOCK as in restore)
+ * Errors also: EXTENT (a slab leaves the pool), HOST_NOT_PINNED, BAD_BLOCK_ID. */
+talaria_status_t talaria_kv_offload_pages(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                          const int32_t *block_table, int64_t first_block,
+                                          int64_t n_blocks, void *host_pool, int64_t pool_bytes,
+                                          const int64_t *page_offsets, void *stream);
+talaria_status_t talaria_kv_restore_pages(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                          const int32_t *new_block_table, int64_t first_block,
+                                          int64_t n_blocks, const void *host_pool, int64_t pool_bytes,
+                                          const int64_t *page_offsets, void *stream);
+
 /* Several sessions in one call (one fused launch per variant where possible). */
 typedef struct {
   const int32_t *block_table; /* HOST */

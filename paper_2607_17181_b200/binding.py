@@ -107,6 +107,8 @@ _SIGNATURES = {
     "talaria_kv_offload": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_restore": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_restore_layered": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P, _P]),
+    "talaria_kv_offload_pages": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.c_int64, _P, _P]),
+    "talaria_kv_restore_pages": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.c_int64, _P, _P]),
     "talaria_kv_gather": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_scatter": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_offload_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
@@ -287,6 +289,18 @@ class Talaria:
         self._check(lib().talaria_kv_restore_layered(self._h, C.byref(kv), _ptr(bt), first_block, n_blocks,
                                                      _ptr(host_src), C.byref(hl), arr, _stream_ptr(stream)),
                     "talaria_kv_restore_layered")
+
+    def kv_offload_pages(self, kv, block_table, first_block, n_blocks, host_pool, pool_bytes, page_offsets, stream=None):
+        bt, po = _i32(block_table), _i64(page_offsets)
+        self._check(lib().talaria_kv_offload_pages(self._h, C.byref(kv), _ptr(bt), first_block, n_blocks,
+                                                   _ptr(host_pool), pool_bytes, _ptr(po), _stream_ptr(stream)),
+                    "talaria_kv_offload_pages")
+
+    def kv_restore_pages(self, kv, new_block_table, first_block, n_blocks, host_pool, pool_bytes, page_offsets, stream=None):
+        bt, po = _i32(new_block_table), _i64(page_offsets)
+        self._check(lib().talaria_kv_restore_pages(self._h, C.byref(kv), _ptr(bt), first_block, n_blocks,
+                                                   _ptr(host_pool), pool_bytes, _ptr(po), _stream_ptr(stream)),
+                    "talaria_kv_restore_pages")
 
     def kv_gather(self, kv, block_table, first_block, n_blocks, d_image, il, stream=None):
         self._kv(lib().talaria_kv_gather, "talaria_kv_gather", kv, block_table, first_block, n_blocks, d_image, il, stream)

@@ -26,6 +26,7 @@ struct KvCopyParams {
   const void *const *plane_base;  // DEVICE [L*P]
   const int32_t *table;           // DEVICE [n], already offset to first_block
   char *img;                      // image base as seen from the device
+  const int64_t *page_off;        // DEVICE [n] or null: extra image offset per logical block
   int64_t sd[3];                  // image stride of digit 0, 1, 2 (bytes)
   int64_t chunk_bytes;
   int64_t w0, w1;                 // chunks [w0, w1) of the image order
@@ -44,6 +45,7 @@ __device__ __forceinline__ void decode_chunk(const KvCopyParams &p, int64_t w, i
   lp = d0 * p.ord.lp_coef[0] + d1 * p.ord.lp_coef[1] + d2 * p.ord.lp_coef[2];
   i = d0 * p.ord.i_coef[0] + d1 * p.ord.i_coef[1] + d2 * p.ord.i_coef[2];
   img_off = d0 * p.sd[0] + d1 * p.sd[1] + d2 * p.sd[2];
+  if (p.page_off) img_off += p.page_off[i];
 }
 
 // 256-bit streaming accesses (sm_100): fewer instructions per byte than 128-bit ones.
@@ -414,6 +416,131 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
 
 
 // ---------------------------------------------------------------------------
+// Page-first registry slabs (App. C): logical block i is one slab of L*P*C bytes,
+// fragments ordered [layer][plane], at byte offset page_off[i] of a pinned host pool.
+// Zero-copy: the copy kernel with one extra offset per block.  Bounce: the dense
+// page-first bounce half is filled / drained by one copy-engine copy per run of
+// adjacent slabs.
+static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const int32_t *table,
+                                          int64_t first, int64_t n, void *host_pool, int64_t pool_bytes,
+                                          const int64_t *page_off, cudaStream_t stream, bool to_image) {
+  if (!kv || first < 0 || n < 0 || pool_bytes < 0) return TALARIA_ERR_INVALID_ARG;
+  if (n == 0) return TALARIA_OK;
+  if (!table || !host_pool || !page_off) return TALARIA_ERR_INVALID_ARG;
+  // a one-block page-first image gives the plan its shape checks and alignment
+  talaria_host_layout_t one{};
+  Plan pl;
+  {
+    const int64_t C0 = (int64_t)kv->num_kv_heads * kv->block_tokens * kv->head_dim * kv->elt_bytes;
+    one.stride_plane = C0;
+    one.stride_layer = (int64_t)kv->num_planes * C0;
+    one.stride_block = (int64_t)kv->num_layers * kv->num_planes * C0;
+    one.capacity_bytes = one.stride_block;
+    TAL_TRY(make_plan(kv, 1, host_pool, &one, &pl));
+  }
+  const int64_t C = pl.C, L = pl.L, P = pl.P, slab = L * P * C;
+  const int32_t *bt = table + first;
+  TAL_TRY(validate_table(ctx, kv, bt, n, /*reject_dups=*/!to_image));
+  uintptr_t bits = 0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (page_off[i] < 0 || page_off[i] + slab > pool_bytes) return TALARIA_ERR_EXTENT;
+    bits |= (uintptr_t)page_off[i];
+  }
+  if (ctx->cfg.validate && to_image) {       // two blocks written into the same slab bytes: order-dependent
+    std::vector<int64_t> sorted(page_off, page_off + n);
+    std::sort(sorted.begin(), sorted.end());
+    for (int64_t i = 1; i < n; ++i)
+      if (sorted[i] < sorted[i - 1] + slab) return TALARIA_ERR_OVERLAP;
+  }
+  int vec = pl.vec;
+  if (bits % 32 != 0 && vec == 32) vec = 16;
+  if (bits % 16 != 0) vec = 0;
+  void *pool_dev;
+  TAL_TRY(mapped_pointer(ctx, host_pool, &pool_dev));
+
+  const size_t ptr_bytes = (size_t)(L * P) * sizeof(void *);
+  const size_t off_bytes = (size_t)n * sizeof(int64_t);
+  const size_t desc_bytes = ptr_bytes + off_bytes + (size_t)n * sizeof(int32_t);
+  DescSlot *slot;
+  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+  memcpy(slot->h, kv->plane_base, ptr_bytes);
+  memcpy(slot->h + ptr_bytes, page_off, off_bytes);
+  memcpy(slot->h + ptr_bytes + off_bytes, bt, (size_t)n * sizeof(int32_t));
+  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+  const int64_t payload = n * slab;
+  ctx->counters.payload_bytes += payload;
+
+  KvCopyParams p{};
+  p.plane_base = (const void *const *)slot->d;
+  p.table = (const int32_t *)(slot->d + ptr_bytes + off_bytes);
+  p.chunk_bytes = C;
+  p.P = (int32_t)P;
+  // digits: plane, layer, block -- the order of bytes inside consecutive slabs
+  p.ord.e0 = P; p.ord.e1 = L;
+  p.ord.lp_coef[0] = 1; p.ord.lp_coef[1] = (int32_t)P; p.ord.lp_coef[2] = 0;
+  p.ord.i_coef[0] = 0; p.ord.i_coef[1] = 0; p.ord.i_coef[2] = 1;
+  p.sd[0] = C; p.sd[1] = P * C;
+
+  BounceLane &ln = ctx->lane[to_image ? 0 : 1];
+  const int64_t dma_min = ctx->cfg.dma_min_bytes > 0 ? ctx->cfg.dma_min_bytes : (8ll << 20);
+  int variant = ctx->cfg.variant;
+  const bool bounce_ok = vec != 0 && (int64_t)ln.half >= slab;
+  if (variant == TALARIA_VARIANT_AUTO || variant == TALARIA_VARIANT_RUNS) {
+    // Measured: for scattered 3 MB slabs the zero-copy kernel (52.7 / 51.5 GB/s) beats one
+    // copy-engine copy per slab (51.9 / 51.2); the copy engine only wins once adjacent slabs
+    // merge into transfers of 16 MiB and more.
+    int64_t runs = 1;
+    for (int64_t i = 1; i < n; ++i)
+      if (page_off[i] != page_off[i - 1] + slab) ++runs;
+    variant = (bounce_ok && payload >= dma_min && payload / runs >= (16ll << 20)) ? TALARIA_VARIANT_BOUNCE
+                                                                                   : TALARIA_VARIANT_ZEROCOPY;
+  }
+  if (variant == TALARIA_VARIANT_BOUNCE && !bounce_ok) variant = TALARIA_VARIANT_ZEROCOPY;
+  ctx->counters.last_variant = variant;
+
+  if (variant == TALARIA_VARIANT_ZEROCOPY) {
+    p.img = (char *)pool_dev;
+    p.page_off = (const int64_t *)(slot->d + ptr_bytes);
+    p.sd[2] = 0;                              // the block's place comes from its page offset
+    p.w0 = 0; p.w1 = n * L * P;
+    TAL_TRY(launch_dir(ctx, to_image, p, vec, zc_grid(ctx), stream));
+    return release_slot(ctx, slot, stream);
+  }
+
+  const int64_t piece = (int64_t)ln.half / slab;          // blocks per bounce half
+  p.page_off = nullptr;
+  p.sd[2] = slab;
+  TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
+  for (int j = 0; j < 2; ++j) TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[j], ln.fork, 0));
+  int k = 0;
+  for (int64_t i0 = 0; i0 < n; i0 += piece, ++k) {
+    const int64_t i1 = std::min(n, i0 + piece);
+    const int j = k & 1;
+    char *half = ln.buf + (size_t)j * ln.half;
+    p.img = half - i0 * slab;
+    p.w0 = i0 * L * P; p.w1 = i1 * L * P;
+    if (to_image) TAL_TRY(launch_dir(ctx, true, p, vec, pack_grid(ctx), ln.s[j]));
+    for (int64_t a = i0; a < i1;) {
+      int64_t b = a + 1;
+      while (b < i1 && page_off[b] == page_off[b - 1] + slab) ++b;
+      char *h = (char *)host_pool + page_off[a];
+      char *d = half + (a - i0) * slab;
+      const size_t bytes = (size_t)((b - a) * slab);
+      if (to_image) TAL_CUDA(ctx, cudaMemcpyAsync(h, d, bytes, cudaMemcpyDeviceToHost, ln.s[j]));
+      else          TAL_CUDA(ctx, cudaMemcpyAsync(d, h, bytes, cudaMemcpyHostToDevice, ln.s[j]));
+      ctx->counters.memcpy_calls++;
+      a = b;
+    }
+    if (!to_image) TAL_TRY(launch_dir(ctx, false, p, vec, pack_grid(ctx), ln.s[j]));
+  }
+  for (int j = 0; j < 2; ++j) {
+    TAL_CUDA(ctx, cudaEventRecord(ln.done[j], ln.s[j]));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[j], 0));
+  }
+  return release_slot(ctx, slot, stream);
+}
+
+// ---------------------------------------------------------------------------
 // Layer-ordered restore (App. C: the layer-first view "matches the device-side KV
 // cache layout used by attention kernels"): the image is brought in layer by
 // layer, whatever its host layout, and an event per layer tells a consumer
@@ -574,6 +701,24 @@ extern "C" talaria_status_t talaria_kv_restore_layered(talaria_ctx *ctx, const t
   TAL_ENTER(ctx);
   return kv_restore_layered(ctx, kv, new_block_table, first_block, n_blocks, host_src, hl, layer_events,
                             (cudaStream_t)stream);
+}
+
+extern "C" talaria_status_t talaria_kv_offload_pages(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                                     const int32_t *block_table, int64_t first_block,
+                                                     int64_t n_blocks, void *host_pool, int64_t pool_bytes,
+                                                     const int64_t *page_offsets, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_transfer_pages(ctx, kv, block_table, first_block, n_blocks, host_pool, pool_bytes, page_offsets,
+                           (cudaStream_t)stream, true);
+}
+
+extern "C" talaria_status_t talaria_kv_restore_pages(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
+                                                     const int32_t *new_block_table, int64_t first_block,
+                                                     int64_t n_blocks, const void *host_pool, int64_t pool_bytes,
+                                                     const int64_t *page_offsets, void *stream) {
+  TAL_ENTER(ctx);
+  return kv_transfer_pages(ctx, kv, new_block_table, first_block, n_blocks, (void *)host_pool, pool_bytes,
+                           page_offsets, (cudaStream_t)stream, false);
 }
 
 extern "C" talaria_status_t talaria_kv_gather(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
