@@ -228,6 +228,28 @@ talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const int32_t *d_c
 int64_t talaria_prefix_agree(int32_t n_ranks, const int64_t *committed_blocks,
                              const uint64_t *hashes, int64_t stride);
 
+/* Host-side page registry (Sec. 4.3: "Each block is keyed by the model name and cumulative
+ * prefix hash, matching the radix tree's chunk granularity").  Maps a chained block hash
+ * (the model key is its seed) to the byte offset of the block's page-first slab in the
+ * pinned host pool.  Pure host code, internally locked; all arrays are HOST arrays.
+ *   insert        : keys already present keep their value (first wins); *n_new (nullable)
+ *                   receives the number of new keys.
+ *   lookup_prefix : number of LEADING hashes that are present; their page offsets are
+ *                   written to page_offsets_out (nullable).  Because the hashes are
+ *                   cumulative, this is the longest restorable prefix of the stream.
+ *   erase         : removes the keys that are present; *n_erased (nullable) counts them.
+ * The table grows by itself. */
+typedef struct talaria_registry talaria_registry;
+talaria_status_t talaria_registry_create(talaria_registry **out, int64_t expected_pages);
+talaria_status_t talaria_registry_destroy(talaria_registry *reg);
+talaria_status_t talaria_registry_insert(talaria_registry *reg, const uint64_t *hashes,
+                                         const int64_t *page_offsets, int64_t n, int64_t *n_new);
+int64_t talaria_registry_lookup_prefix(talaria_registry *reg, const uint64_t *hashes, int64_t n,
+                                       int64_t *page_offsets_out);
+talaria_status_t talaria_registry_erase(talaria_registry *reg, const uint64_t *hashes, int64_t n,
+                                        int64_t *n_erased);
+int64_t talaria_registry_size(talaria_registry *reg);
+
 /* ---- (2)/(3) block-table copies ------------------------------------------- */
 
 /* Sec. 4.3 checkpoint: host_dst[l,p,i] <- pool_{l,p}[block_table[first_block+i]]

@@ -321,3 +321,40 @@ def mark_dirty(staging: np.ndarray, plan, alloc_off: int, alloc_bytes: int, stag
     arr = _plan_array(staging, None, staging, plan)
     return int(lib().orc_mark_dirty(arr, len(plan), staging.ctypes.data + alloc_off, alloc_bytes,
                                     _ptr(staged), _ptr(dirty)))
+
+
+# ---------------------------------------------------------------- registry
+
+
+class Registry:
+    """Plain-dict definition of the page registry (Sec. 4.3: blocks keyed by cumulative
+    prefix hash): first insert wins, lookup_prefix counts the leading hashes present."""
+
+    def __init__(self):
+        self.d = {}
+
+    def insert(self, hashes, page_offsets) -> int:
+        new = 0
+        for h, o in zip(hashes, page_offsets):
+            if int(h) not in self.d:
+                self.d[int(h)] = int(o)
+                new += 1
+        return new
+
+    def lookup_prefix(self, hashes):
+        out = []
+        for h in hashes:
+            if int(h) not in self.d:
+                break
+            out.append(self.d[int(h)])
+        return len(out), np.array(out, dtype=np.int64)
+
+    def erase(self, hashes) -> int:
+        gone = 0
+        for h in hashes:
+            if self.d.pop(int(h), None) is not None:
+                gone += 1
+        return gone
+
+    def __len__(self):
+        return len(self.d)

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libtalaria.so")
-SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "stage.cu"]
+SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "stage.cu", "registry.cu"]
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_BLOCK_ID, ERR_DUP_BLOCK, ERR_HOST_NOT_PINNED = -1, -2, -3, -4
@@ -104,6 +104,12 @@ _SIGNATURES = {
     "talaria_prefix_match_host": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
     "talaria_prefix_match_static": (C.c_int32, [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
     "talaria_prefix_agree": (C.c_int64, [C.c_int32, _P, _P, C.c_int64]),
+    "talaria_registry_create": (C.c_int32, [C.POINTER(_P), C.c_int64]),
+    "talaria_registry_destroy": (C.c_int32, [_P]),
+    "talaria_registry_insert": (C.c_int32, [_P, _P, _P, C.c_int64, C.POINTER(C.c_int64)]),
+    "talaria_registry_lookup_prefix": (C.c_int64, [_P, _P, C.c_int64, _P]),
+    "talaria_registry_erase": (C.c_int32, [_P, _P, C.c_int64, C.POINTER(C.c_int64)]),
+    "talaria_registry_size": (C.c_int64, [_P]),
     "talaria_kv_offload": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_restore": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P]),
     "talaria_kv_restore_layered": (C.c_int32, [_P, C.POINTER(KvLayout), _P, C.c_int64, C.c_int64, _P, C.POINTER(HostLayout), _P, _P]),
@@ -189,6 +195,54 @@ def kv_layout(shape, plane_ptrs: Sequence[int], num_blocks: int):
 
 def host_layout(strides, capacity_bytes: int) -> HostLayout:
     return HostLayout(strides[0], strides[1], strides[2], capacity_bytes)
+
+
+class Registry:
+    """Host-side page registry: chained block hash -> page offset (needs no GPU)."""
+
+    def __init__(self, expected_pages: int = 1024):
+        self._h = C.c_void_p()
+        rc = lib().talaria_registry_create(C.byref(self._h), expected_pages)
+        if rc != OK:
+            raise TalariaError(rc, "talaria_registry_create")
+
+    def insert(self, hashes, page_offsets) -> int:
+        h = np.ascontiguousarray(hashes, dtype=np.uint64)
+        po = _i64(page_offsets)
+        assert h.size == po.size
+        n_new = C.c_int64()
+        rc = lib().talaria_registry_insert(self._h, _ptr(h), _ptr(po), h.size, C.byref(n_new))
+        if rc != OK:
+            raise TalariaError(rc, "talaria_registry_insert")
+        return n_new.value
+
+    def lookup_prefix(self, hashes):
+        h = np.ascontiguousarray(hashes, dtype=np.uint64)
+        out = np.zeros(max(h.size, 1), np.int64)
+        k = int(lib().talaria_registry_lookup_prefix(self._h, _ptr(h), h.size, _ptr(out)))
+        return k, out[:k]
+
+    def erase(self, hashes) -> int:
+        h = np.ascontiguousarray(hashes, dtype=np.uint64)
+        n = C.c_int64()
+        rc = lib().talaria_registry_erase(self._h, _ptr(h), h.size, C.byref(n))
+        if rc != OK:
+            raise TalariaError(rc, "talaria_registry_erase")
+        return n.value
+
+    def __len__(self):
+        return int(lib().talaria_registry_size(self._h))
+
+    def destroy(self):
+        if self._h:
+            lib().talaria_registry_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 class Talaria:

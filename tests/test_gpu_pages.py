@@ -101,3 +101,44 @@ def test_page_argument_errors(ctxs):
     assert status(ctx.kv_offload_pages, pool.kv, [0, 1, 2, 3], 0, 4, np.zeros(8 * slab, np.uint8), 8 * slab, offs) == tb.ERR_HOST_NOT_PINNED
     ctx.kv_restore_pages(pool.kv, [3, 2, 1, 0], 0, 4, host.ptr, host.n, [0, 0, 0, 0])     # reading one slab four times is fine
     ctx.sync()
+
+
+def test_registry_keyed_restore_end_to_end(ctxs):
+    """Turn finishes: pages are checkpointed and registered under their cumulative hashes.  The
+    session returns with a longer prompt: its hashes are computed on the GPU, the registry gives
+    the longest run of pages present, and exactly those pages are restored into new blocks."""
+    ctx = ctxs[tb.VARIANT_AUTO]
+    shape, nb = wl.TINY, 256
+    g = wl.rng(1)
+    wl.tokens(g, 300)
+    sess = wl.tokens(g, 500)
+    cont = wl.continuation(g, sess, 560, 350)
+    planes = wl.kv_pool(g, shape, nb)
+    pool = DevicePool(shape, planes)
+    n_full = 500 // 16
+    src, dst = wl.disjoint_tables(g, nb, [n_full, 560 // 16 + 1])
+    slab = shape.bytes_per_block
+    host = GuardedPinned(64 * slab)
+    offs = g.permutation(64)[:n_full].astype(np.int64) * slab
+    # checkpoint + register (GPU hashes of the stored stream, read back to the host)
+    ctx.kv_offload_pages(pool.kv, src, 0, n_full, host.ptr, host.n, offs)
+    res = np.zeros(1, tb.MATCH_DTYPE)
+    hs = np.zeros(n_full, np.uint64)
+    ctx.prefix_match_host(1, sess, [0, 500], sess[:0], [0, 0], None, 16, wl.HASH_SEED, hs, res)
+    reg, ref = tb.Registry(), orc.Registry()
+    assert reg.insert(hs, offs) == ref.insert(orc.block_hash(sess, 16, wl.HASH_SEED), offs) == n_full
+    # the session returns
+    hc = np.zeros(560 // 16, np.uint64)
+    ctx.prefix_match_host(1, cont, [0, 560], sess, [0, 500], hs, 16, wl.HASH_SEED, hc, res)
+    k, pages = reg.lookup_prefix(hc)
+    k_ref, pages_ref = ref.lookup_prefix(orc.block_hash(cont, 16, wl.HASH_SEED))
+    assert k == k_ref == 21 == int(res[0]["matched_blocks"]) and np.array_equal(pages, pages_ref)
+    ctx.kv_restore_pages(pool.kv, dst, 0, k, host.ptr, host.n, pages)
+    ctx.sync()
+    want_host = np.zeros(host.n, np.uint8)
+    orc.kv_pages(oshape(shape), planes, src, 0, n_full, want_host, offs, True)
+    assert np.array_equal(host.np, want_host)
+    orc.kv_pages(oshape(shape), planes, dst, 0, k_ref, want_host, pages_ref, False)
+    for a, b in zip(pool.read(), planes):
+        assert np.array_equal(a, b)
+    reg.destroy()
