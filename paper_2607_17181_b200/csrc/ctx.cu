@@ -131,6 +131,9 @@ static void destroy_impl(talaria_ctx *ctx) {
     if (s.h) cudaFreeHost(s.h);
     if (s.d) cudaFree(s.d);
   }
+  if (ctx->prefix_busy) cudaEventSynchronize(ctx->prefix_done);
+  if (ctx->prefix_done) cudaEventDestroy(ctx->prefix_done);
+  if (ctx->prefix_counters) cudaFree(ctx->prefix_counters);
   if (ctx->prefix_scratch.p) cudaFree(ctx->prefix_scratch.p);
   if (ctx->host_tok.p) cudaFree(ctx->host_tok.p);
   for (auto &r : ctx->registered) cudaHostUnregister(r.first);
@@ -173,6 +176,9 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
       TAL_CUDA(ctx, cudaMalloc((void **)&s.d, kSlotBytes));
       s.cap = kSlotBytes;
     }
+    TAL_CUDA(ctx, cudaMalloc((void **)&ctx->prefix_counters, 64 * sizeof(unsigned int)));
+    TAL_CUDA(ctx, cudaMemset(ctx->prefix_counters, 0, 64 * sizeof(unsigned int)));
+    TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->prefix_done, cudaEventDisableTiming));
     // Internal streams run at the highest priority: their kernels are short packing
     // steps that gate copy-engine transfers, so they should not queue behind a long
     // kernel of the caller's (for example a staging copy on another stream).

@@ -46,6 +46,10 @@ struct talaria_ctx {
   int ring_next = 0;
   tal::BounceLane lane[tal::kLanes];
   tal::DevBuf prefix_scratch;         // digests + per-tile mismatch positions
+  unsigned int *prefix_counters = nullptr;  // per-pair tile counters of the fused prefix kernel (zero at rest)
+  cudaEvent_t prefix_done = nullptr;  // end of the last prefix call (its scratch is shared)
+  bool prefix_busy = false;
+  cudaStream_t prefix_stream = nullptr;  // stream of that call (same stream: already ordered)
   tal::DevBuf host_tok;               // device copies for talaria_prefix_match_host
   std::vector<std::pair<char *, size_t>> registered;
   std::vector<uint64_t> dup_bits;     // restore-table duplicate check

@@ -4,7 +4,8 @@
 //   digest_k = sum_j mix64(u32(tok[kB+j]) + G*(j+1));  s_k = s_{k-1}*P + digest_k;
 //   hash_k   = mix64(s_k)
 //
-// Two launches per call, whatever the number of pairs:
+// Up to eight pairs (a session returning) run as ONE fused launch: the CTA that finishes a
+// pair's last tile also runs that pair's chain.  Larger batches use two launches:
 //   1. tile kernel  -- a CTA per 2048-token tile of a pair: coalesced 16-byte token
 //      loads (four tokens per thread, summed in registers), a warp-shuffle
 //      segmented sum over the B/4 lanes that share a block, and the first token
@@ -47,6 +48,7 @@ struct PairDesc {
 };
 
 constexpr int kInlinePairs = 8;    // up to this many pairs travel in the kernel parameters
+constexpr int64_t kFusedMaxTiles = 296;    // 2 CTAs per SM x 148 SMs: about one wave of the fused kernel
 
 struct PrefixParams {
   const PairDesc *pairs;      // DEVICE [n_pairs + 1] (last entry holds the totals); null when inline
@@ -63,6 +65,7 @@ struct PrefixParams {
   uint64_t *cont_hashes_out;  // DEVICE or null
   talaria_match_t *results;   // DEVICE [n_pairs] or null
   uint64_t seed;
+  unsigned int *counters;     // DEVICE [kInlinePairs], zero between calls (fused kernel only)
 };
 
 __device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int m) {
@@ -72,7 +75,8 @@ __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
   return (uint64_t)__shfl_up_sync(0xffffffffu, (unsigned long long)v, d);
 }
 
-__global__ void __launch_bounds__(kTileThreads) prefix_tile_kernel(const __grid_constant__ PrefixParams p) {
+// Work of one 2,048-token tile; returns the pair the tile belongs to.
+__device__ __forceinline__ int tile_body(const PrefixParams &p) {
   __shared__ long long s_min[kTileThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   int q = 0;
@@ -200,6 +204,11 @@ __global__ void __launch_bounds__(kTileThreads) prefix_tile_kernel(const __grid_
     for (int k = 1; k < kTileThreads / 32; ++k) v = s_min[k] < v ? s_min[k] : v;
     p.tile_mis[blockIdx.x] = v;
   }
+  return q;
+}
+
+__global__ void __launch_bounds__(kTileThreads) prefix_tile_kernel(const __grid_constant__ PrefixParams p) {
+  (void)tile_body(p);
 }
 
 // (a1,b1) then (a2,b2):  x -> (x*a1 + b1)*a2 + b2
@@ -210,15 +219,14 @@ __device__ __forceinline__ Affine2 then(const Affine2 &f, const Affine2 &g) {
   return Affine2{f.a * g.a, f.bc * g.a + g.bc, f.bs * g.a + g.bs};
 }
 
-__global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid_constant__ PrefixParams p) {
+// Chain, compare and result record of one pair, by one CTA of kScanThreads threads.  Digests and
+// tile results were written by other CTAs, so they are read through L2 (ld.global.cg).
+__device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair) {
   __shared__ Affine2 s_warp[kScanThreads / 32];
   __shared__ uint64_t s_carry[2];
   __shared__ long long s_red[kScanThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  // Launched as a programmatic dependent of the tile kernel: CTAs may be resident early,
-  // and this wait returns once the tile kernel has finished and its writes are visible.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  const PairDesc pd = p.pairs ? p.pairs[blockIdx.x] : p.inl[blockIdx.x];
+  const PairDesc pd = p.pairs ? p.pairs[pair] : p.inl[pair];
   const int B = p.B;
   const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
   const int64_t lim = nbc < nbs ? nbc : nbs;                 // blocks that can be compared
@@ -240,8 +248,8 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
 #pragma unroll
     for (int q = 0; q < kScanItems; ++q) {
       const int64_t k = k0 + q;
-      vc[q] = (k < nbc) ? dc[k] : 0ull;
-      vs[q] = (derive_s && k < nbs) ? ds[k] : 0ull;
+      vc[q] = (k < nbc) ? __ldcg(dc + k) : 0ull;
+      vs[q] = (derive_s && k < nbs) ? __ldcg(ds + k) : 0ull;
       if (k < nb) loc = Affine2{loc.a * kP, loc.bc * kP + vc[q], loc.bs * kP + vs[q]};
     }
     // inclusive scan across the warp
@@ -282,9 +290,9 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
 
   // token-level first mismatch over this pair's tiles
   long long lcp = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
-  const int64_t t0 = pd.tile_off, t1 = p.pairs ? p.pairs[blockIdx.x + 1].tile_off : p.inl[blockIdx.x + 1].tile_off;
+  const int64_t t0 = pd.tile_off, t1 = p.pairs ? p.pairs[pair + 1].tile_off : p.inl[pair + 1].tile_off;
   for (int64_t t = t0 + tid; t < t1; t += kScanThreads) {
-    long long v = p.tile_mis[t];
+    long long v = __ldcg(p.tile_mis + t);
     lcp = v < lcp ? v : lcp;
   }
   for (int m = 16; m >= 1; m >>= 1) {
@@ -311,8 +319,38 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
       r.reusable_tokens = (long long)B * (first_bad < lcp_blocks ? first_bad : lcp_blocks);
       r.hash_token_disagree = (first_bad != tok_blocks) ? 1 : 0;
       r.reserved = 0;
-      p.results[blockIdx.x] = r;
+      p.results[pair] = r;
     }
+  }
+}
+
+__global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid_constant__ PrefixParams p) {
+  // Launched as a programmatic dependent of the tile kernel: CTAs may be resident early,
+  // and this wait returns once the tile kernel has finished and its writes are visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  chain_body(p, (int)blockIdx.x);
+}
+
+// One launch for a handful of pairs (a session returning): every CTA does its tile, and the
+// CTA that finishes a pair's last tile also runs that pair's chain.  Completion is counted with
+// one atomic per CTA; nobody waits for anybody.  The counter is put back to zero by the CTA
+// that saw the last arrival, so the next call finds it clean.
+static_assert(kTileThreads == kScanThreads, "the fused kernel runs both bodies with one block size");
+__global__ void __launch_bounds__(kTileThreads) prefix_fused_kernel(const __grid_constant__ PrefixParams p) {
+  __shared__ int s_last;
+  const int q = tile_body(p);
+  __threadfence();                       // this thread's digests / tile result are visible device-wide
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned tiles_q = (unsigned)(p.inl[q + 1].tile_off - p.inl[q].tile_off);
+    const unsigned prev = atomicAdd(&p.counters[q], 1u);
+    s_last = (prev + 1 == tiles_q);
+    if (s_last) p.counters[q] = 0;
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    chain_body(p, q);
   }
 }
 
@@ -351,19 +389,32 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     big.resize((size_t)n_pairs + 1);
     pd = big.data();
   }
+  // A handful of pairs run as ONE fused launch (every pair then owns at least one tile, so some
+  // CTA always finishes it); big batches keep two lean kernels for throughput.
+  bool fused = inl;
   int64_t cb = 0, sb = 0, tiles = 0;
-  for (int32_t q = 0; q < n_pairs; ++q) {
-    int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
-    if (Tc < 0 || Ts < 0 || cont_off[q] < 0 || sess_off[q] < 0) return TALARIA_ERR_INVALID_ARG;
-    pd[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, tiles};
-    cb += Tc / B;
-    sb += Ts / B;
-    tiles += (std::max(Tc, Ts) + kTileTok - 1) / kTileTok;
+  for (int pass = 0; pass < 2; ++pass) {
+    cb = sb = tiles = 0;
+    for (int32_t q = 0; q < n_pairs; ++q) {
+      int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
+      if (Tc < 0 || Ts < 0 || cont_off[q] < 0 || sess_off[q] < 0) return TALARIA_ERR_INVALID_ARG;
+      pd[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, tiles};
+      cb += Tc / B;
+      sb += Ts / B;
+      const int64_t t = (std::max(Tc, Ts) + kTileTok - 1) / kTileTok;
+      tiles += fused ? std::max<int64_t>(t, 1) : t;
+    }
+    if (!fused || tiles <= kFusedMaxTiles) break;
+    fused = false;                        // too much work for one wave of CTAs: lay out again, unfused
   }
   pd[n_pairs] = PairDesc{cont_off[n_pairs], sess_off[n_pairs], 0, 0, cb, sb, tiles};
   if (cont_off[n_pairs] > cont_off[0] && !d_cont) return TALARIA_ERR_INVALID_ARG;
   if (sess_off[n_pairs] > sess_off[0] && !d_sess) return TALARIA_ERR_INVALID_ARG;
   if (tiles > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
+
+  // The scratch (digests, tile results, counters) is shared by all calls of this context:
+  // a call on another stream must not start before the previous call's kernels are done.
+  if (ctx->prefix_busy && ctx->prefix_stream != stream) TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->prefix_done, 0));
 
   const bool derive = (d_sess_hashes == nullptr);
   const size_t dig_c_bytes = (size_t)cb * 8, dig_s_bytes = derive ? (size_t)sb * 8 : 0;
@@ -400,13 +451,23 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   p.cont_hashes_out = d_cont_hashes;
   p.results = d_results;
   p.seed = seed;
-  if (tiles > 0) {
-    prefix_tile_kernel<<<(unsigned)tiles, kTileThreads, 0, stream>>>(p);
+  p.counters = ctx->prefix_counters;
+  if (fused) {
+    prefix_fused_kernel<<<(unsigned)tiles, kTileThreads, 0, stream>>>(p);
     TAL_CUDA(ctx, cudaGetLastError());
     ctx->counters.kernel_launches++;
+  } else {
+    if (tiles > 0) {
+      prefix_tile_kernel<<<(unsigned)tiles, kTileThreads, 0, stream>>>(p);
+      TAL_CUDA(ctx, cudaGetLastError());
+      ctx->counters.kernel_launches++;
+    }
+    TAL_CUDA(ctx, launch_chain(p, n_pairs, stream));
+    ctx->counters.kernel_launches++;
   }
-  TAL_CUDA(ctx, launch_chain(p, n_pairs, stream));
-  ctx->counters.kernel_launches++;
+  TAL_CUDA(ctx, cudaEventRecord(ctx->prefix_done, stream));
+  ctx->prefix_busy = true;
+  ctx->prefix_stream = stream;
   return slot ? release_slot(ctx, slot, stream) : TALARIA_OK;
 }
 

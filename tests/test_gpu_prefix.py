@@ -185,3 +185,25 @@ def test_bad_arguments(ctx):
         ctx.prefix_match(1, d, [0, 64], d, [64, 0], None, 16, 0, None, out)    # negative length
     ctx.block_hash(d, 64, 16, 0, out)
     ctx.sync()
+
+
+def test_calls_on_two_streams_share_scratch_safely(ctx):
+    # the context's digest scratch is shared: calls on different streams must not overlap on the GPU
+    g = wl.rng(507)
+    jobs = []
+    for k in range(6):
+        s = wl.tokens(g, 60_000 + 1000 * k)
+        c = wl.continuation(g, s, 64_000, 30_000 + 500 * k)
+        jobs.append((c, s, _dev(c), _dev(s), torch.zeros(64_000 // 16, dtype=torch.int64, device="cuda"),
+                     torch.zeros(4, dtype=torch.int64, device="cuda")))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for k, (c, s, dc, ds, dh, dr) in enumerate(jobs):
+            ctx.prefix_match(1, dc, [0, c.size], ds, [0, s.size], None, 16, SEED, dh, dr, stream=streams[k % 3])
+    torch.cuda.synchronize()
+    for c, s, dc, ds, dh, dr in jobs:
+        m, hc = orc.prefix_match(c, s, 16, SEED)
+        r = dr.cpu().numpy()
+        assert [int(r[0]), int(r[1]), int(r[2])] == [m.lcp_tokens, m.matched_blocks, m.reusable_tokens]
+        assert np.array_equal(dh.cpu().numpy().view(np.uint64), hc)
