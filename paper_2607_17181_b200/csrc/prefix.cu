@@ -243,15 +243,20 @@ __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair
 
   for (int64_t chunk = 0; chunk < nb; chunk += (int64_t)kScanThreads * kScanItems) {
     const int64_t k0 = chunk + (int64_t)tid * kScanItems;
-    uint64_t vc[kScanItems], vs[kScanItems];
+    uint64_t vc[kScanItems], vs[kScanItems], hs_st[kScanItems];
     Affine2 loc{1ull, 0ull, 0ull};
+    // all loads of this thread's run are issued up front (the stored hashes too: fetched
+    // inside the compare loop they would serialise behind the hash stores)
 #pragma unroll
     for (int q = 0; q < kScanItems; ++q) {
       const int64_t k = k0 + q;
       vc[q] = (k < nbc) ? __ldcg(dc + k) : 0ull;
       vs[q] = (derive_s && k < nbs) ? __ldcg(ds + k) : 0ull;
-      if (k < nb) loc = Affine2{loc.a * kP, loc.bc * kP + vc[q], loc.bs * kP + vs[q]};
+      hs_st[q] = (!derive_s && k < lim) ? __ldg(hs_in + k) : 0ull;
     }
+#pragma unroll
+    for (int q = 0; q < kScanItems; ++q)
+      if (k0 + q < nb) loc = Affine2{loc.a * kP, loc.bc * kP + vc[q], loc.bs * kP + vs[q]};
     // inclusive scan across the warp
     Affine2 inc = loc;
 #pragma unroll
@@ -278,7 +283,7 @@ __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair
         const uint64_t hc = mix64(sc);
         if (k < nbc && hc_out) hc_out[k] = hc;
         if (k < lim) {
-          const uint64_t hs = derive_s ? mix64(ss) : hs_in[k];
+          const uint64_t hs = derive_s ? mix64(ss) : hs_st[q];
           if (hs != hc && k < first_bad) first_bad = k;
         }
       }
