@@ -70,7 +70,7 @@ typedef struct {
   int32_t variant;        /* TALARIA_VARIANT_*; overridden by env TALARIA_VARIANT=1|2|3       */
   int32_t validate;       /* 0 = skip host-side table / plan validation; default 1            */
   int32_t zc_ctas;        /* grid size of zero-copy kernels; 0 = built-in (leaves SMs free)   */
-  int32_t hbm_ctas_per_sm;/* resident CTAs per SM for HBM-bound kernels; 0 = built-in         */
+  int32_t pack_ctas;      /* grid size of the bounce variant's pack / unpack kernels; 0 = 64  */
 } talaria_config_t;
 
 /* Device-side paged KV pool (Sec. 4.3; descriptor fields of App. C "Attention-layout

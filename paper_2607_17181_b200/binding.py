@@ -46,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 class Config(C.Structure):
     _fields_ = [("bounce_bytes", C.c_int64), ("dma_min_bytes", C.c_int64), ("variant", C.c_int32),
-                ("validate", C.c_int32), ("zc_ctas", C.c_int32), ("hbm_ctas_per_sm", C.c_int32)]
+                ("validate", C.c_int32), ("zc_ctas", C.c_int32), ("pack_ctas", C.c_int32)]
 
 
 class KvLayout(C.Structure):
@@ -249,9 +249,9 @@ class Talaria:
     """One library context on one CUDA device."""
 
     def __init__(self, device: int = 0, variant: int = VARIANT_AUTO, bounce_bytes: int = 0,
-                 dma_min_bytes: int = 0, validate: bool = True, zc_ctas: int = 0, hbm_ctas_per_sm: int = 0):
+                 dma_min_bytes: int = 0, validate: bool = True, zc_ctas: int = 0, pack_ctas: int = 0):
         self._h = C.c_void_p()
-        cfg = Config(bounce_bytes, dma_min_bytes, variant, 1 if validate else 0, zc_ctas, hbm_ctas_per_sm)
+        cfg = Config(bounce_bytes, dma_min_bytes, variant, 1 if validate else 0, zc_ctas, pack_ctas)
         rc = lib().talaria_create(C.byref(self._h), device, C.byref(cfg))
         if rc != OK:
             self._h = C.c_void_p()

@@ -104,11 +104,6 @@ talaria_status_t require_device_pointer(talaria_ctx *ctx, const void *p) {
   return TALARIA_ERR_INVALID_ARG;
 }
 
-int hbm_grid(const talaria_ctx *ctx, int threads_per_cta) {
-  int per_sm = ctx->cfg.hbm_ctas_per_sm > 0 ? ctx->cfg.hbm_ctas_per_sm : std::max(1, 2048 / threads_per_cta);
-  return ctx->sm_count * per_sm;
-}
-
 }  // namespace tal
 
 using namespace tal;

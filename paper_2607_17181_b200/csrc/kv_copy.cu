@@ -6,7 +6,7 @@
 // (fastest-varying dimension first), so the image side of the copy is a single
 // sequential stream -- full 128-byte lines on the host link -- while the pool side
 // jumps from chunk to chunk as the block table says.  Each warp moves 4 KiB per
-// step with eight 16-byte accesses per lane in flight.
+// step, every lane keeping 128 bytes in flight (four 256-bit or eight 128-bit accesses).
 #include <algorithm>
 #include <cstring>
 
@@ -30,7 +30,6 @@ struct KvCopyParams {
   int64_t sd[3];                  // image stride of digit 0, 1, 2 (bytes)
   int64_t chunk_bytes;
   int64_t w0, w1;                 // chunks [w0, w1) of the image order
-  int32_t P;
   ImgOrder ord;
 };
 
@@ -46,24 +45,6 @@ __device__ __forceinline__ void decode_chunk(const KvCopyParams &p, int64_t w, i
   i = d0 * p.ord.i_coef[0] + d1 * p.ord.i_coef[1] + d2 * p.ord.i_coef[2];
   img_off = d0 * p.sd[0] + d1 * p.sd[1] + d2 * p.sd[2];
   if (p.page_off) img_off += p.page_off[i];
-}
-
-// 256-bit streaming accesses (sm_100): fewer instructions per byte than 128-bit ones.
-struct alignas(32) Vec32 {
-  unsigned r[8];
-};
-__device__ __forceinline__ Vec32 ld_cs_32(const void *p) {
-  Vec32 v;
-  asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]),
-                 "=r"(v.r[6]), "=r"(v.r[7])
-               : "l"(p));
-  return v;
-}
-__device__ __forceinline__ void st_cs_32(void *p, const Vec32 &v) {
-  asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]),
-               "r"(v.r[3]), "r"(v.r[4]), "r"(v.r[5]), "r"(v.r[6]), "r"(v.r[7]), "l"(p)
-               : "memory");
 }
 
 // TO_IMAGE: pool -> image (offload / gather); else image -> pool (restore / scatter).
@@ -268,7 +249,7 @@ static void set_image_strides(KvCopyParams &p, const ImgOrder &o, int64_t sL, in
 static int64_t zc_grid(const talaria_ctx *ctx) { return ctx->cfg.zc_ctas > 0 ? ctx->cfg.zc_ctas : 32; }
 // Pack / unpack kernels of the bounce variant only have to stay ahead of a 56 GB/s copy engine;
 // a small grid does that with a 20x margin and barely disturbs concurrent kernels.
-static int64_t pack_grid(const talaria_ctx *ctx) { return 2 * zc_grid(ctx); }
+static int64_t pack_grid(const talaria_ctx *ctx) { return ctx->cfg.pack_ctas > 0 ? ctx->cfg.pack_ctas : 64; }
 // In-HBM gather / scatter: one short CTA per 16 warps of work, scheduled by the hardware.
 static int64_t full_grid() { return 0x7fffffff; }
 
@@ -313,7 +294,6 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
   p.plane_base = (const void *const *)slot->d;
   p.table = (const int32_t *)(slot->d + ptr_bytes);
   p.chunk_bytes = pl.C;
-  p.P = (int32_t)pl.P;
   p.ord = pl.ord;
 
   const int64_t payload = pl.chunks * pl.C;
@@ -474,7 +454,6 @@ static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_lay
   p.plane_base = (const void *const *)slot->d;
   p.table = (const int32_t *)(slot->d + ptr_bytes + off_bytes);
   p.chunk_bytes = C;
-  p.P = (int32_t)P;
   // digits: plane, layer, block -- the order of bytes inside consecutive slabs
   p.ord.e0 = P; p.ord.e1 = L;
   p.ord.lp_coef[0] = 1; p.ord.lp_coef[1] = (int32_t)P; p.ord.lp_coef[2] = 0;
@@ -634,8 +613,7 @@ static talaria_status_t kv_restore_layered(talaria_ctx *ctx, const talaria_kv_la
       p.plane_base = (const void *const *)slot->d + l0 * P;
       p.table = (const int32_t *)(slot->d + ptr_bytes) + i0;
       p.chunk_bytes = C;
-      p.P = (int32_t)P;
-      p.img = half;
+          p.img = half;
       p.w0 = 0;
       p.w1 = LL * P * nn;
       if (rows_by_block) {        // digits: plane, block, layer

@@ -30,23 +30,6 @@ constexpr int kStageThreads = 512;
 constexpr int kStageTile = kStageThreads * 128;      // 64 KiB: 128 bytes in flight per thread
 constexpr int kSpanTiles = 8;                        // tiles per CTA (512 KiB)
 
-struct alignas(32) Vec32 {
-  unsigned r[8];
-};
-__device__ __forceinline__ Vec32 ld_cs_32(const void *p) {
-  Vec32 v;
-  asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(v.r[0]), "=r"(v.r[1]), "=r"(v.r[2]), "=r"(v.r[3]), "=r"(v.r[4]), "=r"(v.r[5]),
-                 "=r"(v.r[6]), "=r"(v.r[7])
-               : "l"(p));
-  return v;
-}
-__device__ __forceinline__ void st_cs_32(void *p, const Vec32 &v) {
-  asm volatile("st.global.cs.v8.b32 [%8], {%0,%1,%2,%3,%4,%5,%6,%7};" ::"r"(v.r[0]), "r"(v.r[1]), "r"(v.r[2]),
-               "r"(v.r[3]), "r"(v.r[4]), "r"(v.r[5]), "r"(v.r[6]), "r"(v.r[7]), "l"(p)
-               : "memory");
-}
-
 struct StageParams {
   const StageEntry *entries;   // DEVICE [n + 1]; entries[n].tile0 = total tiles
   const int32_t *span_entry;   // DEVICE [grid]: entry that holds the span's first tile
