@@ -309,7 +309,8 @@ talaria_status_t talaria_kv_restore_pages(talaria_ctx *ctx, const talaria_kv_lay
                                           int64_t n_blocks, const void *host_pool, int64_t pool_bytes,
                                           const int64_t *page_offsets, void *stream);
 
-/* Several sessions in one call (one fused launch per variant where possible). */
+/* Several sessions in one call: each transfer is enqueued in turn on `stream`; restore tables
+ * are checked against each other first (no block may be claimed twice). */
 typedef struct {
   const int32_t *block_table; /* HOST */
   int64_t first_block, n_blocks;
@@ -371,6 +372,24 @@ talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_copy_t *plan, 
  * number of bits that changed from clean to dirty. */
 int64_t talaria_mark_dirty(const talaria_copy_t *plan, int64_t n, const void *alloc_base,
                            int64_t alloc_bytes, const uint8_t *staged_bitmap, uint8_t *dirty_bitmap);
+
+/* ---- argument checks that need no GPU ------------------------------------------ */
+
+/* The same host-side validation the copy and stage calls apply, callable on its own
+ * (for example when a table or plan is built, long before it is used).
+ *   check_block_table  : BAD_BLOCK_ID, and DUP_BLOCK when reject_duplicates != 0.
+ *   check_image_layout : the three strides must nest without overlap (INVALID_ARG) and the
+ *                        image must fit capacity_bytes (EXTENT); plane_base may be NULL.
+ *                        *contiguous_run_bytes (nullable) receives the length of the image's
+ *                        contiguous runs, which decides whether large copy-engine
+ *                        transfers are possible.
+ *   check_stage_plan   : INVALID_ARG / OVERLAP as in talaria_stage; fills stats. */
+talaria_status_t talaria_check_block_table(const int32_t *block_table, int64_t n, int64_t num_blocks,
+                                           int32_t reject_duplicates);
+talaria_status_t talaria_check_image_layout(const talaria_kv_layout_t *kv, int64_t n_blocks,
+                                            const talaria_host_layout_t *hl, int64_t *contiguous_run_bytes);
+talaria_status_t talaria_check_stage_plan(const talaria_copy_t *plan, int64_t n, const uint8_t *dirty_bitmap,
+                                          talaria_stage_stats_t *stats);
 
 /* ---- completion, errors, counters ------------------------------------------ */
 

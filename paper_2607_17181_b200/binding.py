@@ -122,6 +122,9 @@ _SIGNATURES = {
     "talaria_stage": (C.c_int32, [_P, _P, C.c_int64, _P, C.POINTER(StageStats), _P]),
     "talaria_prestage": (C.c_int32, [_P, _P, C.c_int64, _P, _P, _P, C.POINTER(StageStats), _P]),
     "talaria_mark_dirty": (C.c_int64, [_P, C.c_int64, _P, C.c_int64, _P, _P]),
+    "talaria_check_block_table": (C.c_int32, [_P, C.c_int64, C.c_int64, C.c_int32]),
+    "talaria_check_image_layout": (C.c_int32, [C.POINTER(KvLayout), C.c_int64, C.POINTER(HostLayout), C.POINTER(C.c_int64)]),
+    "talaria_check_stage_plan": (C.c_int32, [_P, C.c_int64, _P, C.POINTER(StageStats)]),
     "talaria_sync": (C.c_int32, [_P, _P]),
     "talaria_strerror": (C.c_char_p, [C.c_int32]),
     "talaria_last_cuda_error": (C.c_int32, [_P]),
@@ -195,6 +198,30 @@ def kv_layout(shape, plane_ptrs: Sequence[int], num_blocks: int):
 
 def host_layout(strides, capacity_bytes: int) -> HostLayout:
     return HostLayout(strides[0], strides[1], strides[2], capacity_bytes)
+
+
+def check_block_table(block_table, num_blocks: int, reject_duplicates: bool) -> int:
+    bt = _i32(block_table)
+    return int(lib().talaria_check_block_table(_ptr(bt), bt.size, num_blocks, 1 if reject_duplicates else 0))
+
+
+def check_image_layout(shape, num_blocks: int, n_blocks: int, strides, capacity_bytes: int):
+    """(status, contiguous run bytes) of an image layout; needs no GPU."""
+    kv = KvLayout(shape.num_layers, shape.num_kv_heads, shape.block_tokens, shape.head_dim, shape.elt_bytes,
+                  shape.num_planes, num_blocks, None)
+    hl = HostLayout(strides[0], strides[1], strides[2], capacity_bytes)
+    run = C.c_int64()
+    rc = int(lib().talaria_check_image_layout(C.byref(kv), n_blocks, C.byref(hl), C.byref(run)))
+    return rc, run.value
+
+
+def check_stage_plan(plan: np.ndarray, dirty_bitmap=None):
+    """(status, StageStats) of a stage plan of COPY_DTYPE entries; needs no GPU."""
+    plan = np.ascontiguousarray(plan, dtype=COPY_DTYPE)
+    bm = None if dirty_bitmap is None else np.ascontiguousarray(dirty_bitmap, dtype=np.uint8)
+    st = StageStats()
+    rc = int(lib().talaria_check_stage_plan(_ptr(plan), plan.size, _ptr(bm), C.byref(st)))
+    return rc, st
 
 
 class Registry:

@@ -120,10 +120,12 @@ struct Plan {
   int vec;             // widest usable access: 32, 16, or 0 (byte path)
 };
 
+// Shape and stride checks, image order, contiguous run length, widest usable access.
+// need_planes = false skips everything that needs the plane addresses (host-only check).
 static talaria_status_t make_plan(const talaria_kv_layout_t *kv, int64_t n, const void *img,
-                                  const talaria_host_layout_t *hl, Plan *out) {
+                                  const talaria_host_layout_t *hl, Plan *out, bool need_planes = true) {
   if (kv->num_layers <= 0 || kv->num_kv_heads <= 0 || kv->block_tokens <= 0 || kv->head_dim <= 0 ||
-      kv->elt_bytes <= 0 || kv->num_planes <= 0 || kv->num_blocks <= 0 || !kv->plane_base)
+      kv->elt_bytes <= 0 || kv->num_planes <= 0 || kv->num_blocks <= 0 || (need_planes && !kv->plane_base))
     return TALARIA_ERR_INVALID_ARG;
   Plan pl{};
   pl.L = kv->num_layers;
@@ -168,7 +170,7 @@ static talaria_status_t make_plan(const talaria_kv_layout_t *kv, int64_t n, cons
   uintptr_t bits = (uintptr_t)pl.C | (uintptr_t)img;    // low bits of everything an address is built from
   for (int k = 0; k < 3; ++k)
     if (d[k].extent != 1) bits |= (uintptr_t)d[k].stride;
-  for (int64_t k = 0; k < pl.L * pl.P; ++k) {
+  for (int64_t k = 0; need_planes && k < pl.L * pl.P; ++k) {
     if (!kv->plane_base[k]) return TALARIA_ERR_INVALID_ARG;
     bits |= (uintptr_t)kv->plane_base[k];
   }
@@ -187,23 +189,26 @@ static int64_t image_offset(const Plan &pl, const talaria_host_layout_t *hl, int
          d[pl.ord.pos_i] * hl->stride_block;
 }
 
-static talaria_status_t validate_table(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const int32_t *bt,
-                                       int64_t n, bool reject_dups) {
-  if (!ctx->cfg.validate) return TALARIA_OK;
-  const int64_t nb = kv->num_blocks;
+static talaria_status_t check_table(const int32_t *bt, int64_t n, int64_t num_blocks, bool reject_dups,
+                                    std::vector<uint64_t> *bits) {
   for (int64_t i = 0; i < n; ++i)
-    if (bt[i] < 0 || (int64_t)bt[i] >= nb) return TALARIA_ERR_BAD_BLOCK_ID;
+    if (bt[i] < 0 || (int64_t)bt[i] >= num_blocks) return TALARIA_ERR_BAD_BLOCK_ID;
   if (reject_dups) {
-    size_t words = (size_t)((nb + 63) / 64);
-    ctx->dup_bits.assign(words, 0);
+    bits->assign((size_t)((num_blocks + 63) / 64), 0);
     for (int64_t i = 0; i < n; ++i) {
-      uint64_t bit = 1ull << (bt[i] & 63);
-      uint64_t &w = ctx->dup_bits[(size_t)bt[i] >> 6];
+      const uint64_t bit = 1ull << (bt[i] & 63);
+      uint64_t &w = (*bits)[(size_t)bt[i] >> 6];
       if (w & bit) return TALARIA_ERR_DUP_BLOCK;
       w |= bit;
     }
   }
   return TALARIA_OK;
+}
+
+static talaria_status_t validate_table(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const int32_t *bt,
+                                       int64_t n, bool reject_dups) {
+  if (!ctx->cfg.validate) return TALARIA_OK;
+  return check_table(bt, n, kv->num_blocks, reject_dups, &ctx->dup_bits);
 }
 
 // vec: access width the addresses allow (0 = byte path); img_bits: low bits of the image base in use.
@@ -653,6 +658,27 @@ using namespace tal;
   std::lock_guard<std::mutex> lk__((ctx)->mu);           \
   DeviceGuard guard__((ctx)->device);                    \
   if (!guard__.ok) return TALARIA_ERR_CUDA
+
+extern "C" talaria_status_t talaria_check_block_table(const int32_t *block_table, int64_t n, int64_t num_blocks,
+                                                      int32_t reject_duplicates) {
+  if (n < 0 || num_blocks <= 0 || (n > 0 && !block_table)) return TALARIA_ERR_INVALID_ARG;
+  std::vector<uint64_t> bits;
+  return check_table(block_table, n, num_blocks, reject_duplicates != 0, &bits);
+}
+
+extern "C" talaria_status_t talaria_check_image_layout(const talaria_kv_layout_t *kv, int64_t n_blocks,
+                                                       const talaria_host_layout_t *hl,
+                                                       int64_t *contiguous_run_bytes) {
+  if (!kv || !hl || n_blocks < 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_blocks == 0) {
+    if (contiguous_run_bytes) *contiguous_run_bytes = 0;
+    return TALARIA_OK;
+  }
+  Plan pl;
+  TAL_TRY(make_plan(kv, n_blocks, nullptr, hl, &pl, /*need_planes=*/false));
+  if (contiguous_run_bytes) *contiguous_run_bytes = pl.run_chunks * pl.C;
+  return TALARIA_OK;
+}
 
 extern "C" talaria_status_t talaria_kv_offload(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
                                                const int32_t *block_table, int64_t first_block,

@@ -113,15 +113,12 @@ static bool cross_overlap(const std::vector<Range> &a, std::vector<Range> &b) {
   return false;
 }
 
-static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
-                                   const uint8_t *dirty, talaria_stage_stats_t *stats, cudaStream_t stream) {
-  if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
+// Which entries come from host, byte / chunk counts, and (optionally) the overlap rules.
+// Needs no GPU: it is also the body of talaria_check_stage_plan.
+static talaria_status_t classify_plan(const talaria_copy_t *plan, int64_t n, const uint8_t *dirty, bool validate,
+                                      std::vector<uint8_t> *from_host_out, int64_t *n_clean_out,
+                                      talaria_stage_stats_t *st_out) {
   talaria_stage_stats_t st{0, 0, 0, 0};
-  if (n == 0) {
-    if (stats) *stats = st;
-    return TALARIA_OK;
-  }
-  // classify
   std::vector<uint8_t> from_host((size_t)n, 0);
   int64_t n_clean = 0;
   for (int64_t k = 0; k < n; ++k) {
@@ -139,7 +136,7 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
       ++n_clean;
     }
   }
-  if (ctx->cfg.validate) {
+  if (validate) {
     std::vector<Range> dsts, srcs;
     dsts.reserve((size_t)n);
     srcs.reserve((size_t)n_clean);
@@ -152,6 +149,23 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
     if (any_overlap_sorted(dsts)) return TALARIA_ERR_OVERLAP;
     if (cross_overlap(dsts, srcs)) return TALARIA_ERR_OVERLAP;
   }
+  if (from_host_out) from_host_out->swap(from_host);
+  if (n_clean_out) *n_clean_out = n_clean;
+  if (st_out) *st_out = st;
+  return TALARIA_OK;
+}
+
+static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                   const uint8_t *dirty, talaria_stage_stats_t *stats, cudaStream_t stream) {
+  if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
+  talaria_stage_stats_t st{0, 0, 0, 0};
+  if (n == 0) {
+    if (stats) *stats = st;
+    return TALARIA_OK;
+  }
+  std::vector<uint8_t> from_host;
+  int64_t n_clean = 0;
+  TAL_TRY(classify_plan(plan, n, dirty, ctx->cfg.validate != 0, &from_host, &n_clean, &st));
 
   // ---- H2D leg, part 1: merge neighbouring host-sourced chunks and check every host
   // source before anything is enqueued, so a rejected plan leaves no partial copy behind.
@@ -292,6 +306,12 @@ extern "C" talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_cop
   tal::DeviceGuard g(ctx->device);
   if (!g.ok) return TALARIA_ERR_CUDA;
   return tal::prestage_impl(ctx, plan, n, blocked_bitmap, staged_bitmap, dirty_bitmap, stats, (cudaStream_t)stream);
+}
+
+extern "C" talaria_status_t talaria_check_stage_plan(const talaria_copy_t *plan, int64_t n,
+                                                     const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats) {
+  if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
+  return tal::classify_plan(plan, n, dirty_bitmap, true, nullptr, nullptr, stats);
 }
 
 extern "C" int64_t talaria_mark_dirty(const talaria_copy_t *plan, int64_t n, const void *alloc_base,
