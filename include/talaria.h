@@ -394,7 +394,11 @@ talaria_status_t talaria_check_stage_plan(const talaria_copy_t *plan, int64_t n,
 /* ---- completion, errors, counters ------------------------------------------ */
 
 /* Sec. 4.3 / App. B "Switch barrier": block the host until everything enqueued on
- * `stream` (offloads included) has finished. */
+ * `stream` (offloads included) has finished.  Also the place where a device-side
+ * finding surfaces: the copy kernels never touch memory outside the pool -- a table
+ * entry outside [0, num_blocks) that reaches them (only possible with validate = 0)
+ * makes them skip that chunk and set a status word, and the next talaria_sync of the
+ * context returns TALARIA_ERR_BAD_BLOCK_ID once (the word is then cleared). */
 talaria_status_t talaria_sync(talaria_ctx *ctx, void *stream);
 
 const char *talaria_strerror(talaria_status_t status);

@@ -53,6 +53,8 @@ struct talaria_ctx {
   tal::DevBuf host_tok;               // device copies for talaria_prefix_match_host
   std::vector<std::pair<char *, size_t>> registered;
   std::vector<uint64_t> dup_bits;     // restore-table duplicate check
+  unsigned int *status_host = nullptr;  // pinned, device-mapped: kernels set it when they skip a bad entry
+  unsigned int *status_dev = nullptr;   // the same word as the device sees it
   int32_t last_cuda_error = 0;
   talaria_counters_t counters{};
 };

@@ -30,6 +30,8 @@ struct KvCopyParams {
   int64_t sd[3];                  // image stride of digit 0, 1, 2 (bytes)
   int64_t chunk_bytes;
   int64_t w0, w1;                 // chunks [w0, w1) of the image order
+  int64_t num_blocks;             // pool capacity: a table entry outside [0, num_blocks) is skipped
+  volatile unsigned int *status;  // device-visible pinned word, set to 1 when an entry was skipped
   ImgOrder ord;
 };
 
@@ -62,6 +64,11 @@ __global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant_
     int64_t lp, i, img_off;
     decode_chunk(p, p.w0 + c, lp, i, img_off);
     int64_t blk = p.table[i];
+    if ((unsigned long long)blk >= (unsigned long long)p.num_blocks) {
+      // never touch memory outside the pool, even when host-side validation was switched off
+      if (lane == 0) *p.status = 1u;
+      continue;
+    }
     char *pool = (char *)p.plane_base[lp] + blk * p.chunk_bytes + part * kPart;
     char *img = p.img + img_off + part * kPart;
     const char *src = TO_IMAGE ? pool : img;
@@ -98,6 +105,10 @@ __global__ void __launch_bounds__(256) kv_copy_byte_kernel(const __grid_constant
     int64_t lp, i, img_off;
     decode_chunk(p, p.w0 + c, lp, i, img_off);
     int64_t blk = p.table[i];
+    if ((unsigned long long)blk >= (unsigned long long)p.num_blocks) {
+      if (lane == 0) *p.status = 1u;
+      continue;
+    }
     char *pool = (char *)p.plane_base[lp] + blk * p.chunk_bytes;
     char *img = p.img + img_off;
     const char *src = TO_IMAGE ? pool : img;
@@ -296,6 +307,8 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
   TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
 
   KvCopyParams p{};
+  p.num_blocks = kv->num_blocks;
+  p.status = ctx->status_dev;
   p.plane_base = (const void *const *)slot->d;
   p.table = (const int32_t *)(slot->d + ptr_bytes);
   p.chunk_bytes = pl.C;
@@ -456,6 +469,8 @@ static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_lay
   ctx->counters.payload_bytes += payload;
 
   KvCopyParams p{};
+  p.num_blocks = kv->num_blocks;
+  p.status = ctx->status_dev;
   p.plane_base = (const void *const *)slot->d;
   p.table = (const int32_t *)(slot->d + ptr_bytes + off_bytes);
   p.chunk_bytes = C;
@@ -615,6 +630,10 @@ static talaria_status_t kv_restore_layered(talaria_ctx *ctx, const talaria_kv_la
       }
       // bounce half -> pool: the half holds [layer][block][plane] or [layer][plane][block]
       KvCopyParams p{};
+      p.num_blocks = kv->num_blocks;
+      p.status = ctx->status_dev;
+  p.num_blocks = kv->num_blocks;
+  p.status = ctx->status_dev;
       p.plane_base = (const void *const *)slot->d + l0 * P;
       p.table = (const int32_t *)(slot->d + ptr_bytes) + i0;
       p.chunk_bytes = C;

@@ -229,3 +229,42 @@ def test_two_streams_offload_and_restore_overlap(ctxs):
     for x, y in zip(pool.read(), planes):
         assert np.array_equal(x, y)
     assert pool.guards_ok() and img_a.guards_ok() and img_b.guards_ok()
+
+
+def test_device_side_guard_skips_bad_entries_when_host_validation_is_off():
+    """With validate=0 a bad table reaches the kernel; it must skip the entry (no access outside the
+    pool), leave everything else exact, and report through talaria_sync.  The bad id used here is
+    num_blocks itself, whose chunk would start right at the end of each plane."""
+    shape, nb = wl.TINY, 16
+    g = wl.rng(19)
+    planes = wl.kv_pool(g, shape, nb)
+    pool = DevicePool(shape, planes)
+    ctx = tb.Talaria(0, variant=tb.VARIANT_ZEROCOPY, validate=False)
+    try:
+        n = 6
+        table = np.array([3, 1, nb, 7, -1, 2], np.int32)              # entries 2 and 4 are outside the pool
+        strides = wl.dense_strides(shape, n, "PF")
+        img = GuardedPinned(n * shape.bytes_per_block, fill=0x99)
+        hl = tb.host_layout(strides, img.n)
+        ctx.kv_offload(pool.kv, table, 0, n, img.ptr, hl)
+        with pytest.raises(tb.TalariaError) as e:
+            ctx.sync()
+        assert e.value.status == tb.ERR_BAD_BLOCK_ID
+        ctx.sync()                                                     # reported once, then clear
+        good = np.array([0, 1, 3, 5])
+        want = np.full(img.n, 0x99, np.uint8)
+        full = np.zeros(img.n, np.uint8)
+        orc.kv_offload(oshape(shape), planes, np.where(table < 0, 0, np.minimum(table, nb - 1)).astype(np.int32),
+                       0, n, full, strides)
+        v_want, v_full = want.reshape(n, -1), full.reshape(n, -1)
+        v_want[good] = v_full[good]                                    # skipped blocks keep the fill
+        assert np.array_equal(img.np, want) and img.guards_ok()
+        # the scatter direction: bad entries are skipped, the pool and its guard bands stay intact
+        ctx.kv_restore(pool.kv, table, 0, n, img.ptr, hl)
+        with pytest.raises(tb.TalariaError):
+            ctx.sync()
+        for a, b in zip(pool.read(), planes):
+            assert np.array_equal(a, b)                               # good entries were restored onto themselves
+        assert pool.guards_ok()
+    finally:
+        ctx.destroy()
