@@ -3,4 +3,4 @@
 The CUDA library is loaded lazily by :mod:`paper_2607_17181_b200.binding`; importing
 the package (for example to reach :mod:`workloads`) does not need a GPU.
 """
-__all__ = ["binding", "workloads"]
+__all__ = ["binding", "workloads", "replay", "replicas", "bench_configs"]
