@@ -207,3 +207,15 @@ def test_calls_on_two_streams_share_scratch_safely(ctx):
         r = dr.cpu().numpy()
         assert [int(r[0]), int(r[1]), int(r[2])] == [m.lcp_tokens, m.matched_blocks, m.reusable_tokens]
         assert np.array_equal(dh.cpu().numpy().view(np.uint64), hc)
+
+
+def test_thousands_of_small_pairs(ctx):
+    # descriptor tables far beyond the inline path, many empty and one-token pairs
+    g = wl.rng(508)
+    pairs = []
+    for _ in range(3000):
+        ts, tc = int(g.integers(0, 300)), int(g.integers(0, 300))
+        s = wl.tokens(g, ts)
+        pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1))), s))
+    _check_batch(ctx, pairs, 16, SEED, False)
+    _check_batch(ctx, pairs, 4, SEED, True)
