@@ -169,7 +169,7 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
     return out
 
 
-def run_replay(torch, dev, ceilings, max_calls=160, host_budget_gb=60.0) -> Dict:
+def run_replay(torch, dev, ceilings, max_calls=160, host_budget_gb=40.0) -> Dict:
     """Session-replay mix at the full KV shape: 30 sessions, pool capped at 60 GB (19,479
     blocks), whole-session LRU eviction to pinned host images, restore on return."""
     shape = wl.QWEN235
@@ -177,17 +177,32 @@ def run_replay(torch, dev, ceilings, max_calls=160, host_budget_gb=60.0) -> Dict
     torch.cuda.empty_cache()
     planes, kv, keep = _pool(torch, dev, shape, pool_blocks, 44)
     ctx = tb.Talaria(dev.index or 0)
-    # one pinned arena, handed out in order and recycled when full (images are dropped on restore)
-    arena = torch.empty(int(host_budget_gb * 1.25e9), dtype=torch.uint8, pin_memory=True)
-    cursor = [0]
+    # one pinned arena with a first-fit free list (pinning is slow; images come and go)
+    arena = torch.empty(int(host_budget_gb * 2e9), dtype=torch.uint8, pin_memory=True)   # 2x: first fit fragments
+    free = [(0, arena.numel())]                     # sorted (offset, length) holes
 
     def alloc_pinned(nbytes):
-        nbytes_al = -(-nbytes // 4096) * 4096
-        if cursor[0] + nbytes_al > arena.numel():
-            cursor[0] = 0
-        t = arena[cursor[0]:cursor[0] + nbytes]
-        cursor[0] += nbytes_al
-        return t
+        need = -(-nbytes // 4096) * 4096
+        fits = [k for k, (_, ln) in enumerate(free) if ln >= need]
+        if not fits:
+            raise MemoryError("pinned arena exhausted")
+        k = min(fits, key=lambda j: free[j][1])          # best fit keeps large holes whole
+        off, ln = free[k]
+        free[k:k + 1] = [(off + need, ln - need)] if ln > need else []
+        return arena[off:off + nbytes]
+
+    def free_pinned(t):
+        off = t.data_ptr() - arena.data_ptr()
+        ln = -(-t.numel() // 4096) * 4096
+        free.append((off, ln))
+        free.sort()
+        merged = []
+        for o, l in free:
+            if merged and merged[-1][0] + merged[-1][1] == o:
+                merged[-1] = (merged[-1][0], merged[-1][1] + l)
+            else:
+                merged.append((o, l))
+        free[:] = merged
 
     scratch = torch.empty(131_072 // 16 * shape.bytes_per_block, dtype=torch.uint8, device=dev)
 
@@ -197,7 +212,7 @@ def run_replay(torch, dev, ceilings, max_calls=160, host_budget_gb=60.0) -> Dict
         return v
 
     drv = ReplayDriver(ctx, shape, kv, pool_blocks, int(host_budget_gb * 1e9), wl.HASH_SEED, content, alloc_pinned,
-                       lambda a: a, order="PF")
+                       lambda a: a, order="PF", free_pinned=free_pinned)
     schedule = wl.session_replay()[:max_calls]
     streams, tg = {}, wl.rng(4, 2)
     groups, cur = [], []

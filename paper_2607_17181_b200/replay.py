@@ -67,13 +67,16 @@ class ReplayStats:
 class ReplayDriver:
     def __init__(self, ctx: tb.Talaria, shape: wl.KvShape, kv, pool_blocks: int, host_budget_bytes: int,
                  seed: int, content: Callable[[int, int, int], np.ndarray], alloc_pinned: Callable[[int], object],
-                 to_device: Callable[[np.ndarray], object], order: str = "PF", log: Optional[list] = None):
+                 to_device: Callable[[np.ndarray], object], order: str = "PF", log: Optional[list] = None,
+                 free_pinned: Optional[Callable[[object], None]] = None):
         """content(session, call_index, nbytes) -> uint8 array: the synthetic KV of a call's new blocks.
-        alloc_pinned(nbytes) -> pinned host tensor; to_device(array) -> device tensor (memory plumbing)."""
+        alloc_pinned(nbytes) -> pinned host tensor; free_pinned(tensor) gives it back (optional);
+        to_device(array) -> device tensor (memory plumbing)."""
         self.ctx, self.shape, self.kv = ctx, shape, kv
         self.pool_blocks, self.host_budget = pool_blocks, host_budget_bytes
         self.seed, self.order = seed, order
         self.content, self.alloc_pinned, self.to_device = content, alloc_pinned, to_device
+        self.free_pinned = free_pinned
         self.free: List[int] = list(range(pool_blocks))      # min-heap: low addresses are reused first
         heapq.heapify(self.free)
         self.sessions: Dict[int, SessionState] = {}
@@ -92,6 +95,8 @@ class ReplayDriver:
 
     def _drop_host(self, s: SessionState):
         self.host_bytes -= s.image_blocks * self.shape.bytes_per_block
+        if self.free_pinned is not None and s.image is not None:
+            self.free_pinned(s.image)
         s.image, s.image_blocks, s.where = None, 0, "none"
 
     def _make_room(self, need: int, busy: set):
