@@ -42,3 +42,11 @@ def test_prefix_agree_needs_no_gpu():
     assert tb.Talaria.prefix_agree([4, 4], h) == 2
     assert tb.Talaria.prefix_agree([1, 4], h) == 1
     assert tb.Talaria.prefix_agree([4], h[:1]) == 4
+
+
+def test_header_is_plain_c(tmp_path):
+    import subprocess
+    src = tmp_path / "hdr.c"
+    src.write_text('#include "talaria.h"\nint main(void) { talaria_match_t m; (void)m; return TALARIA_OK; }\n')
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                           "-I", os.path.join(ROOT, "include"), str(src)])
