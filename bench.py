@@ -210,6 +210,12 @@ def run_other_workload(args):
     elif args.workload == "stage":
         res = bc.run_stage(torch, dev, ceilings, float(peaks["hbm_gbs"]))
         unit = "GB/s read+write of the D2D staging kernel, all chunks clean, alone"
+    elif args.workload == "sweep":
+        res = bc.run_sweep(torch, dev, ceilings)
+        unit = "GB/s best bounce-variant offload of the 25,000-token session"
+    elif args.workload == "prefix":
+        res = bc.run_prefix(torch, dev)
+        unit = "tokens/s, batch of 1,024 pairs x 32,768 tokens, both streams hashed"
     else:
         res = bc.run_replay(torch, dev, ceilings)
         unit = "GB/s aggregate offload+restore payload over the drained transfer calls"
@@ -493,8 +499,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 zero-copy, 2 bounce+DMA, 3 per-run DMA")
     ap.add_argument("--scale", default="full", choices=["full", "small"], help="small = profiling-sized workload")
-    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay"],
-                    help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]")
+    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay", "sweep", "prefix"],
+                    help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]; "
+                         "sweep = variant / size table; prefix = match latency and batch throughput")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

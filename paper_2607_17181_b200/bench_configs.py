@@ -253,3 +253,106 @@ def run_replay(torch, dev, ceilings, max_calls=160, host_budget_gb=40.0) -> Dict
             "timing": "host wall clock around each drained batched call (transfers are 0.1 s and longer)",
             "wall_s_including_host_side_generation": wall,
             "value": (st.offload_bytes + st.restore_bytes) / max(st.offload_s + st.restore_s, 1e-9) / 1e9}
+
+
+def run_sweep(torch, dev, ceilings) -> Dict:
+    """Offload / restore time per variant over transfer sizes (the table behind the AUTO
+    thresholds), the bounce-buffer size sweep, and both directions at once."""
+    shape, NB = wl.QWEN235, 4096
+    planes, kv, keep = _pool(torch, dev, shape, NB, 21)
+    g = wl.rng(2)
+    perm = g.permutation(NB).astype(np.int32)
+    n_max = shape.blocks_for(25_000)
+    bt, bt2 = np.ascontiguousarray(perm[:n_max]), np.ascontiguousarray(perm[n_max:2 * n_max])
+    image = torch.empty(n_max * shape.bytes_per_block, dtype=torch.uint8, pin_memory=True)
+    image2 = torch.empty(n_max * shape.bytes_per_block, dtype=torch.uint8, pin_memory=True)
+    sa, sb = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    rows = []
+    for nblk in (1, 4, 16, 64, 256, 1024, n_max):
+        hl = tb.host_layout(wl.dense_strides(shape, nblk, "PF"), image.numel())
+        row = {"blocks": nblk, "payload_bytes": nblk * shape.bytes_per_block}
+        for variant in (tb.VARIANT_ZEROCOPY, tb.VARIANT_BOUNCE, tb.VARIANT_RUNS):
+            if variant == tb.VARIANT_RUNS and nblk > 256:
+                continue                                    # one 16 KiB copy per chunk: minutes at this size
+            ctx = tb.Talaria(dev.index or 0, variant=variant)
+            reps = 20 if nblk <= 64 else 5
+            row[f"offload_v{variant}_us"] = _timed(torch, sa, lambda: ctx.kv_offload(kv, bt, 0, nblk, image, hl, stream=sa), reps) * 1e3
+            row[f"restore_v{variant}_us"] = _timed(torch, sa, lambda: ctx.kv_restore(kv, bt2, 0, nblk, image, hl, stream=sa), reps) * 1e3
+            ctx.destroy()
+        rows.append(row)
+    hl = tb.host_layout(wl.dense_strides(shape, n_max, "PF"), image.numel())
+    size = image.numel()
+    bounce = []
+    for mib in (32, 64, 128, 256, 512):
+        ctx = tb.Talaria(dev.index or 0, variant=tb.VARIANT_BOUNCE, bounce_bytes=mib << 20)
+        t_o = _timed(torch, sa, lambda: ctx.kv_offload(kv, bt, 0, n_max, image, hl, stream=sa), 5)
+        t_r = _timed(torch, sa, lambda: ctx.kv_restore(kv, bt2, 0, n_max, image, hl, stream=sa), 5)
+        bounce.append({"bounce_mib": mib, "offload_gbs": size / t_o / 1e6, "restore_gbs": size / t_r / 1e6})
+        ctx.destroy()
+    both = []
+    ctxs = {v: tb.Talaria(dev.index or 0, variant=v) for v in (tb.VARIANT_ZEROCOPY, tb.VARIANT_BOUNCE)}
+    for vo in ctxs:
+        for vr in ctxs:
+            best = None
+            for _ in range(3):
+                torch.cuda.synchronize()
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                e[0].record(sa); e[2].record(sb)
+                ctxs[vo].kv_offload(kv, bt, 0, n_max, image, hl, stream=sa); e[1].record(sa)
+                ctxs[vr].kv_restore(kv, bt2, 0, n_max, image2, hl, stream=sb); e[3].record(sb)
+                torch.cuda.synchronize()
+                t = (e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3]))
+                if best is None or max(t) < max(best):
+                    best = t
+            both.append({"offload_variant": vo, "restore_variant": vr, "offload_gbs": size / best[0] / 1e6,
+                         "restore_gbs": size / best[1] / 1e6, "total_gbs": 2 * size / max(best) / 1e6})
+    for c in ctxs.values():
+        c.destroy()
+    return {"workload": "variant sweep: Qwen3-235B KV shape, random block tables, page-first pinned image",
+            "sizes": rows, "bounce_buffer": bounce, "bidirectional": both,
+            "value": max(b["offload_gbs"] for b in bounce)}
+
+
+def run_prefix(torch, dev) -> Dict:
+    """Prefix-match latency for one returning session and throughput for a large batch."""
+    ctx = tb.Talaria(dev.index or 0)
+    g = wl.rng(2)
+    out = {"workload": "prefix match: one pair at session sizes; batch of 1,024 pairs x 32,768 tokens", "single": []}
+    st = torch.cuda.Stream(device=dev)
+    for Ts, Tc, shared in ((25_000, 27_000, 24_000), (105_000, 110_000, 100_000)):
+        sess = wl.tokens(g, Ts)
+        cont = wl.continuation(g, sess, Tc, shared)
+        d_c, d_s = torch.from_numpy(cont).to(dev), torch.from_numpy(sess).to(dev)
+        d_st = torch.empty(Ts // 16, dtype=torch.int64, device=dev)
+        ctx.block_hash(d_s, Ts, 16, wl.HASH_SEED, d_st, stream=st)
+        d_h = torch.empty(Tc // 16, dtype=torch.int64, device=dev)
+        d_r = torch.zeros(4, dtype=torch.int64, device=dev)
+        for stored in (d_st, None):
+            call = lambda: ctx.prefix_match(1, d_c, [0, Tc], d_s, [0, Ts], stored, 16, wl.HASH_SEED, d_h, d_r, stream=st)
+            back = _timed(torch, st, lambda: [call() for _ in range(200)], 3) / 200
+            t0 = time.perf_counter()
+            for _ in range(200):
+                call()
+                ctx.sync(st)
+            lat = (time.perf_counter() - t0) / 200
+            out["single"].append({"cont_tokens": Tc, "sess_tokens": Ts, "stored_hashes": stored is not None,
+                                  "us_per_call_back_to_back": back * 1e3, "us_call_plus_sync_via_python": lat * 1e6})
+    npairs, T = 1024, 32768
+    big_c = torch.randint(0, wl.VOCAB, (npairs * T,), dtype=torch.int32, device=dev)
+    big_s = big_c.clone()
+    big_s[T // 2::T] += 1
+    offs = np.arange(npairs + 1, dtype=np.int64) * T
+    d_hb = torch.empty(npairs * T // 16, dtype=torch.int64, device=dev)
+    d_rb = torch.zeros(npairs * 4, dtype=torch.int64, device=dev)
+    d_stb = torch.zeros(npairs * T // 16, dtype=torch.int64, device=dev)
+    out["batch"] = []
+    for stored in (None, d_stb):
+        ms = _timed(torch, st, lambda: ctx.prefix_match(npairs, big_c, offs, big_s, offs, stored, 16, wl.HASH_SEED,
+                                                        d_hb, d_rb, stream=st), 10)
+        mixes = npairs * T * (2 if stored is None else 1)
+        out["batch"].append({"stored_hashes": stored is not None, "ms": ms, "tokens_per_s": 2 * npairs * T / ms * 1e3,
+                             "token_read_gbs": 2 * npairs * T * 4 / ms / 1e6, "mixes_per_s": mixes / ms * 1e3,
+                             "frac_of_alu_ceiling_1.08e12_mixes_per_s": mixes / ms * 1e3 / 1.08e12})
+    ctx.destroy()
+    out["value"] = out["batch"][0]["tokens_per_s"]
+    return out

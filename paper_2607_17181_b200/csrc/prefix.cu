@@ -25,7 +25,8 @@ namespace tal {
 
 constexpr uint64_t kG = 0x9E3779B97F4A7C15ull;
 constexpr uint64_t kP = 0xD1342543DE82EF95ull;
-constexpr int kTileTok = 2048;
+constexpr int kTileTok = 2048;        // tokens per tile: latency path (fused kernel, static entry point)
+constexpr int kBatchTileTok = 8192;   // tokens per tile in big batches: amortises the per-CTA start-up
 constexpr int kTileThreads = 256;
 constexpr int kScanThreads = 256;
 constexpr int kScanItems = 8;
@@ -58,6 +59,7 @@ struct PrefixParams {
   int32_t B;
   int32_t log2B;              // >= 0 when B is a power of two <= 32, else -1
   int32_t need_sess_digest;   // 1 when stored hashes are not supplied
+  int32_t tile_tok;           // tokens per tile (a multiple of 1024)
   const int32_t *cont, *sess; // DEVICE tokens
   uint64_t *dig_c, *dig_s;    // DEVICE scratch digests
   long long *tile_mis;        // DEVICE scratch [total tiles]
@@ -88,7 +90,8 @@ __device__ __forceinline__ int tile_body(const PrefixParams &p) {
       if (p.inl[k].tile_off <= (int64_t)blockIdx.x) q = k;
   }
   const PairDesc pd = p.pairs ? p.pairs[q] : p.inl[q];
-  const int64_t base = ((int64_t)blockIdx.x - pd.tile_off) * kTileTok;
+  const int tile_tok = p.tile_tok;
+  const int64_t base = ((int64_t)blockIdx.x - pd.tile_off) * tile_tok;
   const int32_t *cont = p.cont + pd.cont_off;
   const int32_t *sess = p.sess + pd.sess_off;
   const int64_t Tmin = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
@@ -101,8 +104,63 @@ __device__ __forceinline__ int tile_body(const PrefixParams &p) {
     // four consecutive tokens per thread (one 16-byte load per stream); the B/4 lanes
     // that share a block finish the sum with xor-shuffles
     const int lanes_per_block = B >> 2;
+    // the position weights of this thread's four tokens never change: rounds advance by a
+    // multiple of the block size
+    const int j_first = (int)((base + (int64_t)tid * 4) & (B - 1));
+    uint64_t wt[4];
 #pragma unroll
-    for (int r = 0; r < kTileTok / (kTileThreads * 4); ++r) {
+    for (int e = 0; e < 4; ++e) wt[e] = kG * (uint64_t)(j_first + e + 1);
+    // interior tile: every token exists in both streams and every block is full, so the
+    // loop carries no bounds checks at all
+    const int64_t tile_end = base + tile_tok;
+    const bool interior = tile_end <= Tmin && tile_end <= nbc * B && (!p.need_sess_digest || tile_end <= nbs * B);
+    if (interior) {
+      const int4 *c4 = (const int4 *)(cont + base) + tid;
+      const int4 *s4 = (const int4 *)(sess + base) + tid;
+      uint64_t *dc = p.dig_c + pd.cont_blk_off + ((base + (int64_t)tid * 4) >> p.log2B);
+      uint64_t *ds = p.dig_s + pd.sess_blk_off + ((base + (int64_t)tid * 4) >> p.log2B);
+      const int blocks_per_round = (kTileThreads * 4) >> p.log2B;
+      const int rounds = tile_tok / (kTileThreads * 4);
+      if (p.need_sess_digest) {
+#pragma unroll 2
+        for (int r = 0; r < rounds; ++r) {
+          const int4 a = __ldg(c4 + r * kTileThreads), b = __ldg(s4 + r * kTileThreads);
+          if ((a.x != b.x) | (a.y != b.y) | (a.z != b.z) | (a.w != b.w)) {
+            const int e = a.x != b.x ? 0 : a.y != b.y ? 1 : a.z != b.z ? 2 : 3;
+            const long long g = base + ((int64_t)r * kTileThreads + tid) * 4 + e;
+            first_mis = g < first_mis ? g : first_mis;
+          }
+          uint64_t vc = mix64((uint64_t)(uint32_t)a.x + wt[0]) + mix64((uint64_t)(uint32_t)a.y + wt[1]) +
+                        mix64((uint64_t)(uint32_t)a.z + wt[2]) + mix64((uint64_t)(uint32_t)a.w + wt[3]);
+          uint64_t vs = mix64((uint64_t)(uint32_t)b.x + wt[0]) + mix64((uint64_t)(uint32_t)b.y + wt[1]) +
+                        mix64((uint64_t)(uint32_t)b.z + wt[2]) + mix64((uint64_t)(uint32_t)b.w + wt[3]);
+          for (int m = 1; m < lanes_per_block; m <<= 1) {
+            vc += shfl_xor_u64(vc, m);
+            vs += shfl_xor_u64(vs, m);
+          }
+          if (j_first == 0) {
+            dc[r * blocks_per_round] = vc;
+            ds[r * blocks_per_round] = vs;
+          }
+        }
+      } else {
+#pragma unroll 2
+        for (int r = 0; r < rounds; ++r) {
+          const int4 a = __ldg(c4 + r * kTileThreads), b = __ldg(s4 + r * kTileThreads);
+          if ((a.x != b.x) | (a.y != b.y) | (a.z != b.z) | (a.w != b.w)) {
+            const int e = a.x != b.x ? 0 : a.y != b.y ? 1 : a.z != b.z ? 2 : 3;
+            const long long g = base + ((int64_t)r * kTileThreads + tid) * 4 + e;
+            first_mis = g < first_mis ? g : first_mis;
+          }
+          uint64_t vc = mix64((uint64_t)(uint32_t)a.x + wt[0]) + mix64((uint64_t)(uint32_t)a.y + wt[1]) +
+                        mix64((uint64_t)(uint32_t)a.z + wt[2]) + mix64((uint64_t)(uint32_t)a.w + wt[3]);
+          for (int m = 1; m < lanes_per_block; m <<= 1) vc += shfl_xor_u64(vc, m);
+          if (j_first == 0) dc[r * blocks_per_round] = vc;
+        }
+      }
+    } else
+#pragma unroll 2
+    for (int r = 0; r < tile_tok / (kTileThreads * 4); ++r) {
       const int64_t g0 = base + ((int64_t)r * kTileThreads + tid) * 4;
       const int64_t k = g0 >> p.log2B;
       const int j0 = (int)(g0 & (B - 1));
@@ -128,9 +186,8 @@ __device__ __forceinline__ int tile_body(const PrefixParams &p) {
       const bool full_c = k < nbc, full_s = p.need_sess_digest && k < nbs;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const uint64_t w = kG * (uint64_t)(j0 + e + 1);
-        if (full_c) vc += mix64((uint64_t)(uint32_t)tc[e] + w);
-        if (full_s) vs += mix64((uint64_t)(uint32_t)ts[e] + w);
+        if (full_c) vc += mix64((uint64_t)(uint32_t)tc[e] + wt[e]);
+        if (full_s) vs += mix64((uint64_t)(uint32_t)ts[e] + wt[e]);
       }
       for (int m = 1; m < lanes_per_block; m <<= 1) {
         vc += shfl_xor_u64(vc, m);
@@ -144,7 +201,7 @@ __device__ __forceinline__ int tile_body(const PrefixParams &p) {
   } else if (p.log2B >= 0) {
     // one token per thread per round; B consecutive lanes own one block
 #pragma unroll 4
-    for (int r = 0; r < kTileTok / kTileThreads; ++r) {
+    for (int r = 0; r < tile_tok / kTileThreads; ++r) {
       const int64_t g = base + r * kTileThreads + tid;
       const int64_t k = g >> p.log2B;
       const int j = (int)(g & (B - 1));
@@ -167,13 +224,13 @@ __device__ __forceinline__ int tile_body(const PrefixParams &p) {
     }
   } else {
     // general block size: a warp per block that STARTS inside this tile
-    for (int r = 0; r < kTileTok / kTileThreads; ++r) {
+    for (int r = 0; r < tile_tok / kTileThreads; ++r) {
       const int64_t g = base + r * kTileThreads + tid;
       if (g < Tmin && first_mis == kNoMismatch && __ldg(cont + g) != __ldg(sess + g)) first_mis = g;
     }
     const int64_t k_first = (base + B - 1) / B;
     const int64_t nb_max = nbc > nbs ? nbc : nbs;
-    for (int64_t k = k_first + wid; k < nb_max && k * B < base + kTileTok; k += kTileThreads / 32) {
+    for (int64_t k = k_first + wid; k < nb_max && k * B < base + tile_tok; k += kTileThreads / 32) {
       const bool dc = k < nbc, ds = p.need_sess_digest && k < nbs;
       uint64_t vc = 0, vs = 0;
       for (int j = lane; j < B; j += 32) {
@@ -398,15 +455,17 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   // CTA always finishes it); big batches keep two lean kernels for throughput.
   bool fused = inl;
   int64_t cb = 0, sb = 0, tiles = 0;
+  int tile_tok = kTileTok;
   for (int pass = 0; pass < 2; ++pass) {
     cb = sb = tiles = 0;
+    tile_tok = fused ? kTileTok : kBatchTileTok;
     for (int32_t q = 0; q < n_pairs; ++q) {
       int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
       if (Tc < 0 || Ts < 0 || cont_off[q] < 0 || sess_off[q] < 0) return TALARIA_ERR_INVALID_ARG;
       pd[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, tiles};
       cb += Tc / B;
       sb += Ts / B;
-      const int64_t t = (std::max(Tc, Ts) + kTileTok - 1) / kTileTok;
+      const int64_t t = (std::max(Tc, Ts) + tile_tok - 1) / tile_tok;
       tiles += fused ? std::max<int64_t>(t, 1) : t;
     }
     if (!fused || tiles <= kFusedMaxTiles) break;
@@ -447,6 +506,7 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     p.log2B = l;
   }
   p.need_sess_digest = derive ? 1 : 0;
+  p.tile_tok = tile_tok;
   p.cont = d_cont;
   p.sess = d_sess;
   p.dig_c = (uint64_t *)ctx->prefix_scratch.p;
@@ -643,6 +703,7 @@ extern "C" talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const i
     p.log2B = l;
   }
   p.need_sess_digest = derive ? 1 : 0;
+  p.tile_tok = kTileTok;
   p.cont = d_cont_tokens;
   p.sess = d_sess_tokens;
   // Every word that is read is written earlier in the same call (digests of full
