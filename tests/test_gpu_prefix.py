@@ -219,3 +219,9 @@ def test_thousands_of_small_pairs(ctx):
         pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1))), s))
     _check_batch(ctx, pairs, 16, SEED, False)
     _check_batch(ctx, pairs, 4, SEED, True)
+
+
+def test_smoke_entry_point_runs():
+    # the build/smoke entry used outside pytest must stay in step with the library
+    import __graft_entry__ as ge
+    ge.smoke()
