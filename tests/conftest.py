@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _native_libraries_present():
+    """Build the CUDA library and the C oracle if a fresh checkout has not done so yet
+    (a no-op when the shared objects are already there)."""
+    from oracle import oracle as orc
+    from paper_2607_17181_b200 import binding as tb
+    if not os.path.exists(tb.LIB_PATH):
+        tb.build()
+    orc.build()
