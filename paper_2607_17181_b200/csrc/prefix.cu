@@ -297,6 +297,16 @@ __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair
   if (tid == 0) { s_carry[0] = p.seed; s_carry[1] = p.seed; }
   __syncthreads();
   long long first_bad = lim;
+  // token-level first mismatch over this pair's tiles: loaded first, so the latency of these
+  // reads overlaps the scan below
+  long long lcp = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
+  {
+    const int64_t t0 = pd.tile_off, t1 = p.pairs ? p.pairs[pair + 1].tile_off : p.inl[pair + 1].tile_off;
+    for (int64_t t = t0 + tid; t < t1; t += kScanThreads) {
+      long long v = __ldcg(p.tile_mis + t);
+      lcp = v < lcp ? v : lcp;
+    }
+  }
 
   for (int64_t chunk = 0; chunk < nb; chunk += (int64_t)kScanThreads * kScanItems) {
     const int64_t k0 = chunk + (int64_t)tid * kScanItems;
@@ -350,13 +360,6 @@ __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair
     __syncthreads();
   }
 
-  // token-level first mismatch over this pair's tiles
-  long long lcp = pd.Tc < pd.Ts ? pd.Tc : pd.Ts;
-  const int64_t t0 = pd.tile_off, t1 = p.pairs ? p.pairs[pair + 1].tile_off : p.inl[pair + 1].tile_off;
-  for (int64_t t = t0 + tid; t < t1; t += kScanThreads) {
-    long long v = __ldcg(p.tile_mis + t);
-    lcp = v < lcp ? v : lcp;
-  }
   for (int m = 16; m >= 1; m >>= 1) {
     long long o = __shfl_xor_sync(0xffffffffu, lcp, m);
     lcp = o < lcp ? o : lcp;
