@@ -213,6 +213,9 @@ def run_other_workload(args):
     elif args.workload == "sweep":
         res = bc.run_sweep(torch, dev, ceilings)
         unit = "GB/s best bounce-variant offload of the 25,000-token session"
+    elif args.workload == "probe":
+        res = bc.run_probe(torch, dev, ceilings)
+        unit = "GB/s read+write, best in-HBM mechanism"
     elif args.workload == "prefix":
         res = bc.run_prefix(torch, dev)
         unit = "tokens/s, batch of 1,024 pairs x 32,768 tokens, both streams hashed"
@@ -499,9 +502,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 zero-copy, 2 bounce+DMA, 3 per-run DMA")
     ap.add_argument("--scale", default="full", choices=["full", "small"], help="small = profiling-sized workload")
-    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay", "sweep", "prefix"],
+    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay", "sweep", "prefix", "probe"],
                     help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]; "
-                         "sweep = variant / size table; prefix = match latency and batch throughput")
+                         "sweep = variant / size table; prefix = match latency and batch throughput; "
+                         "probe = copy mechanisms (128-bit, 256-bit, TMA bulk) vs the copy engine")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

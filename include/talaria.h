@@ -49,7 +49,7 @@ enum {
   TALARIA_ERR_OVERLAP = -6,         /* stage plan: destinations overlap each other or a   */
                                     /* source that is read                                */
   TALARIA_ERR_CUDA = -7,            /* a CUDA call failed: see talaria_last_cuda_error    */
-  TALARIA_ERR_TIMEOUT = -8,         /* reserved: no device-side wait exists on this path  */
+  TALARIA_ERR_TIMEOUT = -8,         /* a bounded device-side wait gave up (probe kernel only) */
   TALARIA_ERR_NO_MEMORY = -9        /* host or device allocation for the context failed   */
 };
 
@@ -390,6 +390,17 @@ talaria_status_t talaria_check_image_layout(const talaria_kv_layout_t *kv, int64
                                             const talaria_host_layout_t *hl, int64_t *contiguous_run_bytes);
 talaria_status_t talaria_check_stage_plan(const talaria_copy_t *plan, int64_t n, const uint8_t *dirty_bitmap,
                                           talaria_stage_stats_t *stats);
+
+/* Copy-mechanism probe (no counterpart in the paper): move `bytes` (a multiple of 16 KiB,
+ * both pointers 32-byte aligned) from src to dst, each DEVICE memory or device-mapped pinned
+ * HOST memory as seen from the device, with one of three mechanisms on `ctas` CTAs:
+ *   0 = 128-bit loads / stores, 1 = 256-bit loads / stores, 2 = TMA bulk copies
+ *   (cp.async.bulk through a four-stage shared-memory ring, no multicast).
+ * Used by `bench.py --workload probe` to show what SM-issued traffic reaches on the host
+ * link and in HBM next to the copy engine.  The TMA variant polls its mbarrier a bounded
+ * number of times; if it ever gives up, the next talaria_sync reports TALARIA_ERR_TIMEOUT. */
+talaria_status_t talaria_probe_copy(talaria_ctx *ctx, int32_t mechanism, const void *src, void *dst,
+                                    int64_t bytes, int32_t ctas, void *stream);
 
 /* ---- completion, errors, counters ------------------------------------------ */
 

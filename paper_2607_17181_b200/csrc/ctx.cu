@@ -243,9 +243,9 @@ extern "C" talaria_status_t talaria_sync(talaria_ctx *ctx, void *stream) {
   TAL_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
   // a copy kernel met a table entry outside the pool (possible only with validation off):
   // it skipped that chunk instead of touching foreign memory; report it once
-  if (*(volatile unsigned int *)ctx->status_host) {
+  if (const unsigned int word = *(volatile unsigned int *)ctx->status_host) {
     *(volatile unsigned int *)ctx->status_host = 0;
-    return TALARIA_ERR_BAD_BLOCK_ID;
+    return (word & 2u) ? TALARIA_ERR_TIMEOUT : TALARIA_ERR_BAD_BLOCK_ID;
   }
   return TALARIA_OK;
 }
