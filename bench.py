@@ -288,7 +288,7 @@ def run_gpu(args):
 
     d_cont = torch.from_numpy(cont).to(dev)
     d_sess = torch.from_numpy(sess).to(dev)
-    ctx = tb.Talaria(local, variant=args.variant)
+    ctx = tb.Talaria(local, variant=args.variant, pack_ctas=args.pack_ctas)
     d_stored = torch.empty(PREFIX_TOKENS // 16, dtype=torch.int64, device=dev)
     ctx.block_hash(d_sess, PREFIX_TOKENS, 16, wl.HASH_SEED, d_stored)     # the registry's stored hashes
     d_hashes = torch.empty(CONT_TOKENS // 16, dtype=torch.int64, device=dev)
@@ -506,6 +506,7 @@ def main():
                     help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]; "
                          "sweep = variant / size table; prefix = match latency and batch throughput; "
                          "probe = copy mechanisms (128-bit, 256-bit, TMA bulk) vs the copy engine")
+    ap.add_argument("--pack-ctas", type=int, default=0, help="grid of the bounce variant's pack kernels (0 = library default)")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
