@@ -75,11 +75,16 @@ __global__ void probe_tma_kernel(const char *__restrict__ src, char *__restrict_
                  : "memory");
   };
   const int64_t ahead = mine < kProbeStages - 1 ? mine : kProbeStages - 1;
-  for (int64_t it = 0; it < ahead; ++it) load(it);
+  int64_t issued = 0;
+  for (; issued < ahead; ++issued) load(issued);
   for (int64_t it = 0; it < mine; ++it) {
     const int s = (int)(it % kProbeStages);
     if (!mbar_wait_bounded(smem_addr(&bars[s]), (uint32_t)((it / kProbeStages) & 1))) {
-      *status = 2u;      // gave up waiting for a load: report, drain what is in flight, leave
+      // gave up waiting for a load: report it, give the other loads in flight one more bounded
+      // wait each (they target this CTA's shared memory), then drain the stores and leave
+      *status = 2u;
+      for (int64_t j = it + 1; j < issued; ++j)
+        (void)mbar_wait_bounded(smem_addr(&bars[j % kProbeStages]), (uint32_t)((j / kProbeStages) & 1));
       break;
     }
     char *g = dst + (first + it * stride) * (int64_t)kProbeChunk;
@@ -87,9 +92,10 @@ __global__ void probe_tma_kernel(const char *__restrict__ src, char *__restrict_
                  "r"(smem_addr(ring + (size_t)s * kProbeChunk)), "r"(kProbeChunk)
                  : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-    if (it + kProbeStages - 1 < mine) {
+    if (issued < mine) {
       asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the previous store has read its stage
-      load(it + kProbeStages - 1);
+      load(issued);
+      ++issued;
     }
   }
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
