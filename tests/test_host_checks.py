@@ -102,3 +102,16 @@ def test_stage_plan_verdicts_against_the_oracle_definition():
     assert tb.check_stage_plan(bad)[0] == tb.ERR_INVALID_ARG          # missing chunk without a host copy
     bad[0] = (base, 0, 0, 16, 0, 0)
     assert tb.check_stage_plan(bad)[0] == tb.ERR_INVALID_ARG          # no destination
+
+
+def test_prefix_agreement_against_the_oracle():
+    # App. B "Prefix agreement": pure host arithmetic, so it is checked here without a GPU
+    g = wl.rng(962)
+    for _ in range(300):
+        R, nb = int(g.integers(1, 9)), int(g.integers(0, 14))
+        hashes = np.tile(g.integers(0, 2**63, size=nb, dtype=np.uint64), (R, 1)) if nb else np.zeros((R, 0), np.uint64)
+        committed = g.integers(0, nb + 1, size=R)
+        for _ in range(int(g.integers(0, 3))):
+            if nb:
+                hashes[int(g.integers(0, R)), int(g.integers(0, nb))] ^= np.uint64(1)
+        assert tb.Talaria.prefix_agree(committed, hashes) == orc.prefix_agree(committed, hashes)
