@@ -349,6 +349,23 @@ talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int
                                const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
                                void *stream);
 
+/* The same switch with the planning taken off the critical path.  A cold-pool instance switches
+ * among a fixed set of models, so the gather plan of a model is known long before the switch
+ * (Sec. 4.4: staging happens "while the current model is serving").  create validates the
+ * plan once (destinations pairwise disjoint and disjoint from EVERY staged source, whatever
+ * a later bitmap says) and keeps its descriptors in device memory; run then costs one bitmap
+ * upload, one launch and the copy-engine copies of the chunks that are dirty or missing this
+ * time.  Results and stats are those of talaria_stage with the same plan and bitmap.  The
+ * bitmap must cover the largest chunk_id of the plan.  Runs of one prepared plan must be
+ * ordered on the GPU by the caller (same stream, or events). */
+typedef struct talaria_stage_plan talaria_stage_plan;
+talaria_status_t talaria_stage_plan_create(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                           talaria_stage_plan **out);
+talaria_status_t talaria_stage_plan_run(talaria_ctx *ctx, talaria_stage_plan *prepared,
+                                        const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
+                                        void *stream);
+talaria_status_t talaria_stage_plan_destroy(talaria_ctx *ctx, talaria_stage_plan *prepared);
+
 /* Sec. 4.4 pre-staging, the step that runs while the current model is still serving:
  * for every plan entry, the authoritative HOST bytes (src_host, pinned) are written to
  * the chunk's place in the staging region (src_dev, a DEVICE address inside unused KV

@@ -143,6 +143,19 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
         bitmap = np.packbits(dirty, bitorder="little")
         h2d = int(sum(plan[k][1] for k in idx))
         t_alone = _timed(torch, sa, lambda: ctx.stage(arr, bitmap, stream=sa), reps)
+        prepared = ctx.stage_plan_create(arr)
+        t_prepared = _timed(torch, sa, lambda: ctx.stage_plan_run(prepared, bitmap, stream=sa), reps)
+        t0 = time.perf_counter()
+        for _ in range(5):
+            ctx.stage_plan_run(prepared, bitmap, stream=sa)
+        host_us_prepared = (time.perf_counter() - t0) / 5 * 1e6
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(5):
+            ctx.stage(arr, bitmap, stream=sa)
+        host_us_plain = (time.perf_counter() - t0) / 5 * 1e6
+        torch.cuda.synchronize()
+        ctx.stage_plan_destroy(prepared)
         t_res_alone = _timed(torch, sb, lambda: ctx.kv_restore(kv, table, 0, nblk, image, hl, stream=sb), reps)
         both = []
         for _ in range(reps):
@@ -157,7 +170,9 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
         d2d = total - h2d
         out["cases"].append({
             "dirty_fraction": frac, "d2d_bytes": d2d, "h2d_bytes": h2d,
-            "stage_alone_ms": t_alone, "stage_with_restore_ms": t_st,
+            "stage_alone_ms": t_alone, "stage_prepared_plan_alone_ms": t_prepared,
+            "host_us_per_call_plain": host_us_plain, "host_us_per_call_prepared": host_us_prepared,
+            "stage_with_restore_ms": t_st,
             "d2d_gbs_read_write_alone": (2 * d2d / t_alone / 1e6) if frac == 0 else None,
             "frac_of_hbm_peak_alone": (2 * d2d / t_alone / 1e6 / hbm_peak) if frac == 0 else None,
             "h2d_gbs_alone": (h2d / t_alone / 1e6) if h2d else None,

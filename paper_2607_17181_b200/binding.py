@@ -120,6 +120,9 @@ _SIGNATURES = {
     "talaria_kv_offload_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
     "talaria_kv_restore_batch": (C.c_int32, [_P, C.POINTER(KvLayout), C.POINTER(KvXfer), C.c_int32, _P]),
     "talaria_stage": (C.c_int32, [_P, _P, C.c_int64, _P, C.POINTER(StageStats), _P]),
+    "talaria_stage_plan_create": (C.c_int32, [_P, _P, C.c_int64, C.POINTER(_P)]),
+    "talaria_stage_plan_run": (C.c_int32, [_P, _P, _P, C.POINTER(StageStats), _P]),
+    "talaria_stage_plan_destroy": (C.c_int32, [_P, _P]),
     "talaria_prestage": (C.c_int32, [_P, _P, C.c_int64, _P, _P, _P, C.POINTER(StageStats), _P]),
     "talaria_mark_dirty": (C.c_int64, [_P, C.c_int64, _P, C.c_int64, _P, _P]),
     "talaria_check_block_table": (C.c_int32, [_P, C.c_int64, C.c_int64, C.c_int32]),
@@ -415,6 +418,23 @@ class Talaria:
         self._check(lib().talaria_stage(self._h, _ptr(plan), plan.size, _ptr(bm), C.byref(st),
                                         _stream_ptr(stream)), "talaria_stage")
         return st
+
+    def stage_plan_create(self, plan: np.ndarray):
+        """Validate and upload a switch plan once; returns an opaque handle for stage_plan_run."""
+        plan = np.ascontiguousarray(plan, dtype=COPY_DTYPE)
+        h = C.c_void_p()
+        self._check(lib().talaria_stage_plan_create(self._h, _ptr(plan), plan.size, C.byref(h)), "talaria_stage_plan_create")
+        return h
+
+    def stage_plan_run(self, prepared, dirty_bitmap: Optional[np.ndarray] = None, stream=None) -> StageStats:
+        bm = None if dirty_bitmap is None else np.ascontiguousarray(dirty_bitmap, dtype=np.uint8)
+        st = StageStats()
+        self._check(lib().talaria_stage_plan_run(self._h, prepared, _ptr(bm), C.byref(st), _stream_ptr(stream)),
+                    "talaria_stage_plan_run")
+        return st
+
+    def stage_plan_destroy(self, prepared):
+        self._check(lib().talaria_stage_plan_destroy(self._h, prepared), "talaria_stage_plan_destroy")
 
     def prestage(self, plan: np.ndarray, blocked_bitmap, staged_bitmap: np.ndarray, dirty_bitmap: np.ndarray,
                  stream=None) -> StageStats:

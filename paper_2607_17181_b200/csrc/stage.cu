@@ -20,10 +20,12 @@
 namespace tal {
 
 struct StageEntry {
-  const char *src;
+  const char *src;  // null: the chunk has no staged copy (always host-sourced)
   char *dst;
   int64_t bytes;
   int64_t tile0;    // first tile of this entry
+  int32_t chunk_id; // bit index into the dirty bitmap, or -1
+  int32_t pad;
 };
 
 constexpr int kStageThreads = 512;
@@ -35,7 +37,13 @@ struct StageParams {
   const int32_t *span_entry;   // DEVICE [grid]: entry that holds the span's first tile
   int64_t n;
   int64_t tiles;
+  const uint8_t *dirty;        // DEVICE bitmap or null (prepared plans): dirty entries are left to the host leg
 };
+
+__device__ __forceinline__ bool stage_skip(const StageParams &p, const StageEntry &e) {
+  if (!e.src) return true;
+  return p.dirty && e.chunk_id >= 0 && ((p.dirty[e.chunk_id >> 3] >> (e.chunk_id & 7)) & 1);
+}
 
 __global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_constant__ StageParams p) {
   const int tid = threadIdx.x;
@@ -44,12 +52,15 @@ __global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_
   int64_t e = p.span_entry[blockIdx.x];
   StageEntry cur = p.entries[e];
   int64_t next_tile0 = p.entries[e + 1].tile0;
+  bool skip = stage_skip(p, cur);
   for (int64_t t = t_begin; t < t_end; ++t) {
     while (t >= next_tile0) {            // entries with zero tiles are skipped too
       ++e;
       cur = p.entries[e];
       next_tile0 = p.entries[e + 1].tile0;
+      skip = stage_skip(p, cur);
     }
+    if (skip) continue;
     const int64_t off = (t - cur.tile0) * kStageTile;
     const int64_t len = min((int64_t)kStageTile, cur.bytes - off);
     const char *src = cur.src + off;
@@ -211,15 +222,15 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
     for (int64_t k = 0; k < n; ++k) {
       if (from_host[(size_t)k]) continue;
       const int64_t nt = (plan[k].bytes + kStageTile - 1) / kStageTile;
-      e[m] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, t0};
+      e[m] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, t0, -1, 0};
       // spans whose first tile falls inside this entry
       while (next_span < spans && next_span * kSpanTiles < t0 + nt) span_entry[next_span++] = (int32_t)m;
       t0 += nt;
       ++m;
     }
-    e[m] = StageEntry{nullptr, nullptr, 0, tiles};
+    e[m] = StageEntry{nullptr, nullptr, 0, tiles, -1, 0};
     TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
-    StageParams p{(const StageEntry *)slot->d, (const int32_t *)(slot->d + ent_bytes), m, tiles};
+    StageParams p{(const StageEntry *)slot->d, (const int32_t *)(slot->d + ent_bytes), m, tiles, nullptr};
     stage_copy_kernel<<<(unsigned)spans, kStageThreads, 0, stream>>>(p);
     TAL_CUDA(ctx, cudaGetLastError());
     ctx->counters.kernel_launches++;
@@ -227,6 +238,158 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   }
   // ---- H2D leg, part 2: enqueued second, so the kernel is already running meanwhile
   if (forked) {
+    for (const HostRun &r : runs) {
+      TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
+      ctx->counters.memcpy_calls++;
+    }
+    TAL_CUDA(ctx, cudaEventRecord(ln.done[0], ln.s[0]));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[0], 0));
+  }
+  ctx->counters.payload_bytes += st.d2d_bytes + st.h2d_bytes;
+  if (stats) *stats = st;
+  return TALARIA_OK;
+}
+
+}  // namespace tal
+
+// A prepared switch plan: validated once, descriptors resident in device memory.  Running it
+// costs one small bitmap upload, one launch and the copy-engine copies of the chunks that are
+// dirty or missing this time; nothing is re-planned on the host.
+struct talaria_stage_plan {
+  std::vector<talaria_copy_t> plan;
+  std::vector<uint8_t> host_pinned;   // per entry: its host copy was found pinned when the plan was made
+  char *d_desc = nullptr;        // entries, then one int32 per span
+  size_t ent_bytes = 0;
+  int64_t tiles = 0, spans = 0, max_chunk = -1;
+  static constexpr int kBitmapRing = 4;
+  uint8_t *d_dirty = nullptr;    // device copy of the bitmap of the current run
+  uint8_t *h_dirty = nullptr;    // pinned staging for it: kBitmapRing buffers used in turn
+  size_t bitmap_bytes = 0;
+  cudaEvent_t uploaded[kBitmapRing] = {};
+  bool busy[kBitmapRing] = {};
+  int next = 0;
+};
+
+namespace tal {
+
+static void plan_free(talaria_stage_plan *sp) {
+  if (!sp) return;
+  for (int r = 0; r < talaria_stage_plan::kBitmapRing; ++r) {
+    if (sp->busy[r]) cudaEventSynchronize(sp->uploaded[r]);
+    if (sp->uploaded[r]) cudaEventDestroy(sp->uploaded[r]);
+  }
+  if (sp->d_desc) cudaFree(sp->d_desc);
+  if (sp->d_dirty) cudaFree(sp->d_dirty);
+  if (sp->h_dirty) cudaFreeHost(sp->h_dirty);
+  (void)cudaGetLastError();
+  delete sp;
+}
+
+static talaria_status_t plan_create(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n, talaria_stage_plan **out) {
+  if (!out || n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
+  *out = nullptr;
+  // validate as if every staged source could be read (whatever the bitmap of a later run says)
+  TAL_TRY(classify_plan(plan, n, nullptr, true, nullptr, nullptr, nullptr));
+  talaria_stage_plan *sp = new (std::nothrow) talaria_stage_plan();
+  if (!sp) return TALARIA_ERR_NO_MEMORY;
+  talaria_status_t st = [&]() -> talaria_status_t {
+    sp->plan.assign(plan, plan + n);
+    sp->host_pinned.assign((size_t)n, 0);
+    for (int64_t k = 0; k < n; ++k) {
+      sp->tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
+      if (plan[k].chunk_id > sp->max_chunk) sp->max_chunk = plan[k].chunk_id;
+      void *alias;
+      if (plan[k].src_host && mapped_pointer(ctx, plan[k].src_host, &alias) == TALARIA_OK) sp->host_pinned[(size_t)k] = 1;
+    }
+    sp->spans = (sp->tiles + kSpanTiles - 1) / kSpanTiles;
+    if (sp->spans > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
+    sp->ent_bytes = ((size_t)(n + 1) * sizeof(StageEntry) + 15) & ~(size_t)15;
+    const size_t desc_bytes = sp->ent_bytes + (size_t)std::max<int64_t>(sp->spans, 1) * sizeof(int32_t);
+    std::vector<char> host(desc_bytes);
+    StageEntry *e = (StageEntry *)host.data();
+    int32_t *span_entry = (int32_t *)(host.data() + sp->ent_bytes);
+    int64_t t0 = 0, next_span = 0;
+    for (int64_t k = 0; k < n; ++k) {
+      const int64_t nt = (plan[k].bytes + kStageTile - 1) / kStageTile;
+      e[k] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, t0, plan[k].chunk_id, 0};
+      while (next_span < sp->spans && next_span * kSpanTiles < t0 + nt) span_entry[next_span++] = (int32_t)k;
+      t0 += nt;
+    }
+    e[n] = StageEntry{nullptr, nullptr, 0, sp->tiles, -1, 0};
+    TAL_CUDA(ctx, cudaMalloc((void **)&sp->d_desc, desc_bytes));
+    TAL_CUDA(ctx, cudaMemcpy(sp->d_desc, host.data(), desc_bytes, cudaMemcpyHostToDevice));
+    sp->bitmap_bytes = (size_t)((sp->max_chunk + 8) / 8);
+    if (sp->bitmap_bytes) {
+      TAL_CUDA(ctx, cudaMalloc((void **)&sp->d_dirty, sp->bitmap_bytes));
+      TAL_CUDA(ctx, cudaHostAlloc((void **)&sp->h_dirty, sp->bitmap_bytes * talaria_stage_plan::kBitmapRing,
+                                  cudaHostAllocDefault));
+    }
+    for (int r = 0; r < talaria_stage_plan::kBitmapRing; ++r)
+      TAL_CUDA(ctx, cudaEventCreateWithFlags(&sp->uploaded[r], cudaEventDisableTiming));
+    return TALARIA_OK;
+  }();
+  if (st != TALARIA_OK) {
+    plan_free(sp);
+    return st;
+  }
+  *out = sp;
+  return TALARIA_OK;
+}
+
+static talaria_status_t plan_run(talaria_ctx *ctx, talaria_stage_plan *sp, const uint8_t *dirty,
+                                 talaria_stage_stats_t *stats, cudaStream_t stream) {
+  if (!sp) return TALARIA_ERR_INVALID_ARG;
+  const int64_t n = (int64_t)sp->plan.size();
+  talaria_stage_stats_t st{0, 0, 0, 0};
+  struct HostRun { const char *h; char *d; int64_t bytes; };
+  std::vector<HostRun> runs;
+  for (int64_t k = 0; k < n; ++k) {
+    const talaria_copy_t &c = sp->plan[k];
+    const bool missing = (c.src_dev == nullptr);
+    const bool is_dirty = !missing && dirty && c.chunk_id >= 0 && ((dirty[c.chunk_id >> 3] >> (c.chunk_id & 7)) & 1);
+    if (!(missing || is_dirty)) {
+      st.d2d_bytes += c.bytes;
+      continue;
+    }
+    if (!c.src_host) return TALARIA_ERR_INVALID_ARG;
+    st.h2d_bytes += c.bytes;
+    if (missing) st.missing_chunks++; else st.dirty_chunks++;
+    if (c.bytes == 0) continue;
+    if (!runs.empty() && runs.back().h + runs.back().bytes == (const char *)c.src_host &&
+        runs.back().d + runs.back().bytes == (char *)c.dst_dev) {
+      runs.back().bytes += c.bytes;
+    } else {
+      if (!sp->host_pinned[(size_t)k]) return TALARIA_ERR_HOST_NOT_PINNED;
+      runs.push_back(HostRun{(const char *)c.src_host, (char *)c.dst_dev, c.bytes});
+    }
+  }
+  const uint8_t *d_bitmap = nullptr;
+  if (dirty && sp->bitmap_bytes) {
+    const int r = sp->next;
+    sp->next = (sp->next + 1) % talaria_stage_plan::kBitmapRing;
+    if (sp->busy[r]) TAL_CUDA(ctx, cudaEventSynchronize(sp->uploaded[r]));   // this pinned buffer is free again
+    uint8_t *h = sp->h_dirty + (size_t)r * sp->bitmap_bytes;
+    memcpy(h, dirty, sp->bitmap_bytes);
+    TAL_CUDA(ctx, cudaMemcpyAsync(sp->d_dirty, h, sp->bitmap_bytes, cudaMemcpyHostToDevice, stream));
+    TAL_CUDA(ctx, cudaEventRecord(sp->uploaded[r], stream));            // h may be rewritten after this
+    sp->busy[r] = true;
+    ctx->counters.memcpy_calls++;
+    d_bitmap = sp->d_dirty;
+  }
+  BounceLane &ln = ctx->lane[1];
+  if (!runs.empty()) {
+    TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
+  }
+  if (sp->tiles > 0 && st.d2d_bytes > 0) {
+    StageParams p{(const StageEntry *)sp->d_desc, (const int32_t *)(sp->d_desc + sp->ent_bytes), n, sp->tiles, d_bitmap};
+    stage_copy_kernel<<<(unsigned)sp->spans, kStageThreads, 0, stream>>>(p);
+    TAL_CUDA(ctx, cudaGetLastError());
+    ctx->counters.kernel_launches++;
+  }
+  // (the device bitmap is rewritten by the next run's upload, which the caller orders after
+  // this kernel: runs of one prepared plan share a stream or are chained with events)
+  if (!runs.empty()) {
     for (const HostRun &r : runs) {
       TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
       ctx->counters.memcpy_calls++;
@@ -306,6 +469,33 @@ extern "C" talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_cop
   tal::DeviceGuard g(ctx->device);
   if (!g.ok) return TALARIA_ERR_CUDA;
   return tal::prestage_impl(ctx, plan, n, blocked_bitmap, staged_bitmap, dirty_bitmap, stats, (cudaStream_t)stream);
+}
+
+extern "C" talaria_status_t talaria_stage_plan_create(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                                      talaria_stage_plan **out) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  tal::DeviceGuard g(ctx->device);
+  if (!g.ok) return TALARIA_ERR_CUDA;
+  return tal::plan_create(ctx, plan, n, out);
+}
+
+extern "C" talaria_status_t talaria_stage_plan_run(talaria_ctx *ctx, talaria_stage_plan *prepared,
+                                                   const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
+                                                   void *stream) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  tal::DeviceGuard g(ctx->device);
+  if (!g.ok) return TALARIA_ERR_CUDA;
+  return tal::plan_run(ctx, prepared, dirty_bitmap, stats, (cudaStream_t)stream);
+}
+
+extern "C" talaria_status_t talaria_stage_plan_destroy(talaria_ctx *ctx, talaria_stage_plan *prepared) {
+  if (!ctx || !prepared) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  tal::DeviceGuard g(ctx->device);
+  tal::plan_free(prepared);
+  return TALARIA_OK;
 }
 
 extern "C" talaria_status_t talaria_check_stage_plan(const talaria_copy_t *plan, int64_t n,

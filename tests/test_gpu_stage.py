@@ -187,3 +187,53 @@ def test_prestage_errors(ctx):
     with pytest.raises(tb.TalariaError) as e:
         ctx.prestage(arr, None, bm, bm.copy())
     assert e.value.status == tb.ERR_INVALID_ARG
+
+
+def test_prepared_plan_runs_match_the_oracle_for_changing_bitmaps(ctx):
+    """One prepared plan, several switches: all clean, 1 % dirty, 36 % dirty, all dirty; some chunks
+    were never staged.  Every run must leave the slots as the oracle's stage() does."""
+    sizes = [300_000, 70_001, 5, 1 << 20, 33_333, 4096 * 192 * 2, 64]
+    plan, total = wl.stage_plan(sizes, 64 << 10)
+    g = wl.rng(602)
+    n = len(plan)
+    weights = g.integers(0, 256, size=total, dtype=np.uint8)
+    missing = g.uniform(size=n) < 0.05
+    host = GuardedPinned(total); host.np[:] = weights
+    staging = GuardedDevice(total, weights)
+    slots = GuardedDevice(total, np.zeros(total, np.uint8))
+    arr = np.zeros(n, tb.COPY_DTYPE)
+    for k, (off, nb, cid) in enumerate(plan):
+        arr[k] = (0 if missing[k] else staging.ptr + off, host.ptr + off, slots.ptr + off, nb, cid, 0)
+    prepared = ctx.stage_plan_create(arr)
+    try:
+        for frac in (0.0, 0.01, 0.36, 1.0, 0.0):
+            dirty = g.uniform(size=n) < frac
+            staged = weights.copy()
+            for (off, nb, cid) in plan:
+                if dirty[cid]:
+                    staged[off:off + nb] ^= 0x5A                    # a KV allocation scribbled over these chunks
+            staging.write(staged)
+            slots.write(np.full(total, 0xEE, np.uint8))
+            bitmap = np.packbits(dirty, bitorder="little")
+            st = ctx.stage_plan_run(prepared, bitmap if frac else None if not dirty.any() else bitmap)
+            ctx.sync()
+            o_slots = np.full(total, 0xEE, np.uint8)
+            entries = [(None if missing[c] else off, off, off, nb, c) for off, nb, c in plan]
+            ost = orc.stage(staged, weights, o_slots, entries, bitmap)
+            assert np.array_equal(slots.read(), o_slots), frac
+            assert (st.d2d_bytes, st.h2d_bytes, st.dirty_chunks, st.missing_chunks) == \
+                (ost.d2d_bytes, ost.h2d_bytes, ost.dirty_chunks, ost.missing_chunks)
+            # and the one-shot call agrees with the prepared one
+            slots.write(np.full(total, 0xEE, np.uint8))
+            ctx.stage(arr, bitmap)
+            ctx.sync()
+            assert np.array_equal(slots.read(), o_slots)
+        assert slots.guards_ok() and staging.guards_ok()
+    finally:
+        ctx.stage_plan_destroy(prepared)
+    bad = arr[:2].copy()
+    bad[1]["dst_dev"] = bad[0]["dst_dev"]
+    bad[1]["bytes"] = bad[0]["bytes"] = 1024
+    with pytest.raises(tb.TalariaError) as e:
+        ctx.stage_plan_create(bad)
+    assert e.value.status == tb.ERR_OVERLAP
