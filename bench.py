@@ -5,7 +5,8 @@ One step = one pass of the whole path for one Qwen3-235B-shaped session
 (94 layers, 4 KV heads, head_dim 128, bf16, 16-token blocks, 25,000-token prefix):
 
     stream A: KV offload of the session's 1,563 scattered blocks to pinned host
-    stream B: D2D staging of a ~59 GB weight set into stable slots   (concurrent)
+    stream B: D2D staging of a ~59 GB weight set into stable slots   (concurrent; the plan was
+              validated and uploaded once, before the timed region: talaria_stage_plan_run)
     drain both (switch barrier)
     prefix match of the 27,000-token continuation (24,000 shared) + result read-back
     KV restore of the matched 1,500 blocks into a different free-block permutation
@@ -289,6 +290,8 @@ def run_gpu(args):
     d_cont = torch.from_numpy(cont).to(dev)
     d_sess = torch.from_numpy(sess).to(dev)
     ctx = tb.Talaria(local, variant=args.variant, pack_ctas=args.pack_ctas)
+    # the model's gather plan is known long before the switch: validate and upload it once
+    prepared = ctx.stage_plan_create(plan_arr) if len(plan_arr) else None
     d_stored = torch.empty(PREFIX_TOKENS // 16, dtype=torch.int64, device=dev)
     ctx.block_hash(d_sess, PREFIX_TOKENS, 16, wl.HASH_SEED, d_stored)     # the registry's stored hashes
     d_hashes = torch.empty(CONT_TOKENS // 16, dtype=torch.int64, device=dev)
@@ -313,7 +316,7 @@ def run_gpu(args):
         if record: m["offload"][1].record(sa)
         if len(plan_arr):
             if record: m["stage"][0].record(sb)
-            ctx.stage(plan_arr, None, stream=sb)
+            ctx.stage_plan_run(prepared, None, stream=sb)
             if record: m["stage"][1].record(sb)
         ctx.sync(sa); ctx.sync(sb)                                   # switch barrier: drain D2H and D2D
         if record: m["match"][0].record(sa)
@@ -388,12 +391,12 @@ def run_gpu(args):
     stage_alone_ms = None
     if len(plan_arr):
         for _ in range(2):
-            ctx.stage(plan_arr, None)
+            ctx.stage_plan_run(prepared, None)
         torch.cuda.synchronize()
         g0, g1 = ev(), ev()
         g0.record()
         for _ in range(5):
-            ctx.stage(plan_arr, None)
+            ctx.stage_plan_run(prepared, None)
         g1.record()
         torch.cuda.synchronize()
         stage_alone_ms = g0.elapsed_time(g1) / 5
