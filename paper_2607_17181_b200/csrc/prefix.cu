@@ -278,6 +278,7 @@ __device__ __forceinline__ Affine2 then(const Affine2 &f, const Affine2 &g) {
 
 // Chain, compare and result record of one pair, by one CTA of kScanThreads threads.  Digests and
 // tile results were written by other CTAs, so they are read through L2 (ld.global.cg).
+template <bool DERIVE_S>
 __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair) {
   __shared__ Affine2 s_warp[kScanThreads / 32];
   __shared__ uint64_t s_carry[2];
@@ -287,7 +288,7 @@ __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair
   const int B = p.B;
   const int64_t nbc = pd.Tc / B, nbs = pd.Ts / B;
   const int64_t lim = nbc < nbs ? nbc : nbs;                 // blocks that can be compared
-  const bool derive_s = p.need_sess_digest != 0;
+  constexpr bool derive_s = DERIVE_S;   // compile-time: the unused stream's registers disappear
   const int64_t nb = derive_s ? (nbc > nbs ? nbc : nbs) : nbc;  // blocks to chain
   const uint64_t *dc = p.dig_c + pd.cont_blk_off;
   const uint64_t *ds = derive_s ? p.dig_s + pd.sess_blk_off : nullptr;
@@ -393,7 +394,8 @@ __global__ void __launch_bounds__(kScanThreads) prefix_chain_kernel(const __grid
   // Launched as a programmatic dependent of the tile kernel: CTAs may be resident early,
   // and this wait returns once the tile kernel has finished and its writes are visible.
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  chain_body(p, (int)blockIdx.x);
+  if (p.need_sess_digest) chain_body<true>(p, (int)blockIdx.x);
+  else                    chain_body<false>(p, (int)blockIdx.x);
 }
 
 // One launch for a handful of pairs (a session returning): every CTA does its tile, and the
@@ -415,7 +417,8 @@ __global__ void __launch_bounds__(kTileThreads) prefix_fused_kernel(const __grid
   __syncthreads();
   if (s_last) {
     __threadfence();
-    chain_body(p, q);
+    if (p.need_sess_digest) chain_body<true>(p, q);
+    else                    chain_body<false>(p, q);
   }
 }
 
