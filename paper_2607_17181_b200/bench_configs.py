@@ -295,6 +295,24 @@ def run_sweep(torch, dev, ceilings) -> Dict:
             row[f"restore_v{variant}_us"] = _timed(torch, sa, lambda: ctx.kv_restore(kv, bt2, 0, nblk, image, hl, stream=sa), reps) * 1e3
             ctx.destroy()
         rows.append(row)
+    # table shape: adjacent ids (one long run) and isolated ids, layer-first image, every variant + AUTO
+    shapes = []
+    hl_lf = tb.host_layout(wl.dense_strides(shape, n_max, "LF"), image.numel())
+    tables = {"random": (bt, bt2),
+              "contiguous": (np.arange(100, 100 + n_max, dtype=np.int32), np.arange(2000, 2000 + n_max, dtype=np.int32)),
+              "isolated": (wl.isolated_table(wl.rng(2, 7), NB, n_max), wl.isolated_table(wl.rng(2, 8), NB, n_max))}
+    for name, (ta, tb_) in tables.items():
+        row = {"table": name, "host_layout": "LF", "blocks": n_max}
+        for variant in (tb.VARIANT_AUTO, tb.VARIANT_ZEROCOPY, tb.VARIANT_BOUNCE, tb.VARIANT_RUNS):
+            if variant == tb.VARIANT_RUNS and name != "contiguous":
+                continue
+            ctx = tb.Talaria(dev.index or 0, variant=variant)
+            t_o = _timed(torch, sa, lambda: ctx.kv_offload(kv, ta, 0, n_max, image, hl_lf, stream=sa), 3)
+            t_r = _timed(torch, sa, lambda: ctx.kv_restore(kv, tb_, 0, n_max, image, hl_lf, stream=sa), 3)
+            row[f"v{variant}"] = {"offload_gbs": image.numel() / t_o / 1e6, "restore_gbs": image.numel() / t_r / 1e6,
+                                  "used": int(ctx.get_counters().last_variant)}
+            ctx.destroy()
+        shapes.append(row)
     hl = tb.host_layout(wl.dense_strides(shape, n_max, "PF"), image.numel())
     size = image.numel()
     bounce = []
@@ -324,7 +342,7 @@ def run_sweep(torch, dev, ceilings) -> Dict:
     for c in ctxs.values():
         c.destroy()
     return {"workload": "variant sweep: Qwen3-235B KV shape, random block tables, page-first pinned image",
-            "sizes": rows, "bounce_buffer": bounce, "bidirectional": both,
+            "sizes": rows, "table_shapes": shapes, "bounce_buffer": bounce, "bidirectional": both,
             "value": max(b["offload_gbs"] for b in bounce)}
 
 
