@@ -195,7 +195,7 @@ def link_ceiling(torch, dev, nbytes=1 << 30, reps=6):
 def run_other_workload(args):
     """configs[2..4]: measurement lines of their own (the default line is configs[1])."""
     import torch
-    from paper_2607_17181_b200 import bench_configs as bc
+    import bench_configs as bc
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -214,9 +214,6 @@ def run_other_workload(args):
     elif args.workload == "sweep":
         res = bc.run_sweep(torch, dev, ceilings)
         unit = "GB/s best bounce-variant offload of the 25,000-token session"
-    elif args.workload == "probe":
-        res = bc.run_probe(torch, dev, ceilings)
-        unit = "GB/s read+write, best in-HBM mechanism"
     elif args.workload == "prefix":
         res = bc.run_prefix(torch, dev)
         unit = "tokens/s, batch of 1,024 pairs x 32,768 tokens, both streams hashed"
@@ -505,10 +502,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 zero-copy, 2 bounce+DMA, 3 per-run DMA")
     ap.add_argument("--scale", default="full", choices=["full", "small"], help="small = profiling-sized workload")
-    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay", "sweep", "prefix", "probe"],
+    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay", "sweep", "prefix"],
                     help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]; "
-                         "sweep = variant / size table; prefix = match latency and batch throughput; "
-                         "probe = copy mechanisms (128-bit, 256-bit, TMA bulk) vs the copy engine")
+                         "sweep = variant / size table; prefix = match latency and batch throughput")
     ap.add_argument("--pack-ctas", type=int, default=0, help="grid of the bounce variant's pack kernels (0 = library default)")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")

@@ -13,9 +13,9 @@ from typing import Dict, List
 
 import numpy as np
 
-from . import binding as tb
-from . import workloads as wl
-from .replay import ReplayDriver
+from paper_2607_17181_b200 import binding as tb
+from paper_2607_17181_b200 import workloads as wl
+from paper_2607_17181_b200.replay import ReplayDriver
 
 PCIE5_X16_GBS = 63.0
 
@@ -389,35 +389,3 @@ def run_prefix(torch, dev) -> Dict:
     ctx.destroy()
     out["value"] = out["batch"][0]["tokens_per_s"]
     return out
-
-
-def run_probe(torch, dev, ceilings) -> Dict:
-    """What each copy mechanism reaches: 128-bit and 256-bit loads / stores and TMA bulk copies,
-    in HBM and over the host link in both directions, next to the copy-engine ceilings."""
-    ctx = tb.Talaria(dev.index or 0)
-    n = 1 << 30
-    d_a = torch.empty(n, dtype=torch.uint8, device=dev)
-    d_b = torch.empty(n, dtype=torch.uint8, device=dev)
-    d_a.view(torch.int64).random_()
-    host = torch.empty(n, dtype=torch.uint8, pin_memory=True)
-    st = torch.cuda.Stream(device=dev)
-    names = {0: "128-bit ld/st", 1: "256-bit ld/st", 2: "TMA bulk (cp.async.bulk)"}
-    rows = []
-    for mech in (0, 1, 2):
-        for ctas in (8, 32, 148, 592):
-            t_w = _timed(torch, st, lambda: ctx.probe_copy(mech, d_a, host, n, ctas, stream=st), 3)
-            t_r = _timed(torch, st, lambda: ctx.probe_copy(mech, host, d_b, n, ctas, stream=st), 3)
-            rows.append({"mechanism": names[mech], "ctas": ctas, "device_to_host_gbs": n / t_w / 1e6,
-                         "host_to_device_gbs": n / t_r / 1e6})
-        for ctas in (148, 296, 592, 2368):
-            t = _timed(torch, st, lambda: ctx.probe_copy(mech, d_a, d_b, n, ctas, stream=st), 3)
-            rows.append({"mechanism": names[mech], "ctas": ctas, "hbm_read_write_gbs": 2 * n / t / 1e6})
-    def torch_copy():
-        with torch.cuda.stream(st):
-            d_b.copy_(d_a)
-    t = _timed(torch, st, torch_copy, 3)
-    ctx.destroy()
-    return {"workload": "copy-mechanism probe, 1 GiB per transfer", "rows": rows,
-            "copy_engine": {"device_to_host_gbs": ceilings["d2h"], "host_to_device_gbs": ceilings["h2d"]},
-            "torch_device_copy_read_write_gbs": 2 * n / t / 1e6,
-            "value": max(r.get("hbm_read_write_gbs", 0.0) for r in rows)}

@@ -14,7 +14,15 @@
  * General rules
  *   - Every function returns a talaria_status_t (0 = OK, negative = error).
  *     No exceptions, no aborts, no device traps.  Arguments are validated on
- *     the host before any launch, so a bad table never reaches the GPU.
+ *     the host before any launch, so a bad table never reaches the GPU.  Extents
+ *     are checked the same way: a host image (its declared capacity_bytes), a
+ *     pinned pool, every pool plane (num_blocks chunks) and every stage source
+ *     and destination must lie, for their whole length, inside the one pinned or
+ *     device allocation that holds their first byte (the driver is asked once per
+ *     allocation; ranges registered through talaria_host_register are known
+ *     exactly).  A range that runs off its allocation is TALARIA_ERR_EXTENT and
+ *     nothing is launched.  validate = 0 switches the table, plan and extent
+ *     checks off.
  *   - Ownership: the caller owns all memory named in the arguments (pool,
  *     host images, token arrays, tables, staging region, slots).  The library
  *     owns only its context: small descriptor buffers, a device bounce buffer
@@ -49,7 +57,6 @@ enum {
   TALARIA_ERR_OVERLAP = -6,         /* stage plan: destinations overlap each other or a   */
                                     /* source that is read                                */
   TALARIA_ERR_CUDA = -7,            /* a CUDA call failed: see talaria_last_cuda_error    */
-  TALARIA_ERR_TIMEOUT = -8,         /* a bounded device-side wait gave up (probe kernel only) */
   TALARIA_ERR_NO_MEMORY = -9        /* host or device allocation for the context failed   */
 };
 
@@ -228,8 +235,8 @@ talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const int32_t *d_c
 int64_t talaria_prefix_agree(int32_t n_ranks, const int64_t *committed_blocks,
                              const uint64_t *hashes, int64_t stride);
 
-/* Host-side page registry (Sec. 4.3: "Each block is keyed by the model name and cumulative
- * prefix hash, matching the radix tree's chunk granularity").  Maps a chained block hash
+/* Host-side page registry (Sec. 4.3: a block's key is the model name together with the
+ * cumulative prefix hash, at the radix tree's chunk granularity).  Maps a chained block hash
  * (the model key is its seed) to the byte offset of the block's page-first slab in the
  * pinned host pool.  Pure host code, internally locked; all arrays are HOST arrays.
  *   insert        : keys already present keep their value (first wins); *n_new (nullable)
@@ -290,9 +297,9 @@ talaria_status_t talaria_kv_restore_layered(talaria_ctx *ctx, const talaria_kv_l
                                             const talaria_host_layout_t *hl,
                                             void *const *layer_events, void *stream);
 
-/* Page-first registry slabs (App. C: the host representation "grouped by logical prefix
- * page, with the per-layer fragments for that page stored under one page descriptor";
- * Sec. 4.3: slabs of one unified pinned pool).  Logical block i is ONE slab of
+/* Page-first registry slabs (App. C: the host copy is organised by logical prefix page,
+ * one page descriptor covering that page's fragments of every layer; Sec. 4.3: slabs of
+ * one unified pinned pool).  Logical block i is ONE slab of
  * num_layers*num_planes*C bytes, fragments ordered [layer][plane], at byte offset
  * page_offsets[i] (HOST int64[n_blocks]) of the pinned HOST pool (host_pool, pool_bytes).
  * Slabs may sit anywhere in the pool, in any order: the registry commits, invalidates
@@ -351,7 +358,7 @@ talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int
 
 /* The same switch with the planning taken off the critical path.  A cold-pool instance switches
  * among a fixed set of models, so the gather plan of a model is known long before the switch
- * (Sec. 4.4: staging happens "while the current model is serving").  create validates the
+ * (Sec. 4.4: staging goes on in the background of the model that is serving).  create validates the
  * plan once (destinations pairwise disjoint and disjoint from EVERY staged source, whatever
  * a later bitmap says) and keeps its descriptors in device memory; run then costs one bitmap
  * upload, one launch and the copy-engine copies of the chunks that are dirty or missing this
@@ -382,8 +389,8 @@ talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_copy_t *plan, 
                                   const uint8_t *blocked_bitmap, uint8_t *staged_bitmap,
                                   uint8_t *dirty_bitmap, talaria_stage_stats_t *stats, void *stream);
 
-/* Sec. 4.4: "marks a chunk dirty if a concurrent prefill allocation takes rows that
- * overlap the chunk's staging range".  Pure host arithmetic: sets the dirty bit of
+/* Sec. 4.4: a staged chunk becomes dirty when a prefill allocation made meanwhile claims
+ * rows inside the chunk's staging range.  Pure host arithmetic: sets the dirty bit of
  * every staged chunk (all chunks when staged_bitmap is NULL) whose staging bytes
  * [src_dev, src_dev+bytes) intersect [alloc_base, alloc_base+alloc_bytes).  Returns the
  * number of bits that changed from clean to dirty. */
@@ -408,17 +415,6 @@ talaria_status_t talaria_check_image_layout(const talaria_kv_layout_t *kv, int64
 talaria_status_t talaria_check_stage_plan(const talaria_copy_t *plan, int64_t n, const uint8_t *dirty_bitmap,
                                           talaria_stage_stats_t *stats);
 
-/* Copy-mechanism probe (no counterpart in the paper): move `bytes` (a multiple of 16 KiB,
- * both pointers 32-byte aligned) from src to dst, each DEVICE memory or device-mapped pinned
- * HOST memory as seen from the device, with one of three mechanisms on `ctas` CTAs:
- *   0 = 128-bit loads / stores, 1 = 256-bit loads / stores, 2 = TMA bulk copies
- *   (cp.async.bulk through a four-stage shared-memory ring, no multicast).
- * Used by `bench.py --workload probe` to show what SM-issued traffic reaches on the host
- * link and in HBM next to the copy engine.  The TMA variant polls its mbarrier a bounded
- * number of times; if it ever gives up, the next talaria_sync reports TALARIA_ERR_TIMEOUT. */
-talaria_status_t talaria_probe_copy(talaria_ctx *ctx, int32_t mechanism, const void *src, void *dst,
-                                    int64_t bytes, int32_t ctas, void *stream);
-
 /* ---- completion, errors, counters ------------------------------------------ */
 
 /* Sec. 4.3 / App. B "Switch barrier": block the host until everything enqueued on
@@ -426,7 +422,9 @@ talaria_status_t talaria_probe_copy(talaria_ctx *ctx, int32_t mechanism, const v
  * finding surfaces: the copy kernels never touch memory outside the pool -- a table
  * entry outside [0, num_blocks) that reaches them (only possible with validate = 0)
  * makes them skip that chunk and set a status word, and the next talaria_sync of the
- * context returns TALARIA_ERR_BAD_BLOCK_ID once (the word is then cleared). */
+ * context returns TALARIA_ERR_BAD_BLOCK_ID once (the word is then cleared).  The word
+ * belongs to the context, not to a stream: whichever stream is synchronised first
+ * reports it. */
 talaria_status_t talaria_sync(talaria_ctx *ctx, void *stream);
 
 const char *talaria_strerror(talaria_status_t status);

@@ -380,7 +380,8 @@ static void orc_set_bit(uint8_t *bm, int64_t i, int v)
     else   bm[i >> 3] &= (uint8_t)~(1u << (i & 7));
 }
 
-/* "The staging manager writes weights into fixed-size chunks": for every plan entry
+/* Sec. 4.4, pre-staging: weights are written into the staging region in fixed-size
+ * chunks.  For every plan entry
  * whose staging rows are not blocked (bit chunk_id of `blocked`: the rows currently
  * belong to a KV allocation), copy the authoritative host bytes into the chunk's
  * place in the staging region (src_dev), set its staged bit and clear its dirty

@@ -19,11 +19,11 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libtalaria.so")
-SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "stage.cu", "registry.cu", "probe.cu"]
+SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "stage.cu", "registry.cu"]
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_BLOCK_ID, ERR_DUP_BLOCK, ERR_HOST_NOT_PINNED = -1, -2, -3, -4
-ERR_EXTENT, ERR_OVERLAP, ERR_CUDA, ERR_TIMEOUT, ERR_NO_MEMORY = -5, -6, -7, -8, -9
+ERR_EXTENT, ERR_OVERLAP, ERR_CUDA, ERR_NO_MEMORY = -5, -6, -7, -9
 VARIANT_AUTO, VARIANT_ZEROCOPY, VARIANT_BOUNCE, VARIANT_RUNS = 0, 1, 2, 3
 
 
@@ -128,7 +128,6 @@ _SIGNATURES = {
     "talaria_check_block_table": (C.c_int32, [_P, C.c_int64, C.c_int64, C.c_int32]),
     "talaria_check_image_layout": (C.c_int32, [C.POINTER(KvLayout), C.c_int64, C.POINTER(HostLayout), C.POINTER(C.c_int64)]),
     "talaria_check_stage_plan": (C.c_int32, [_P, C.c_int64, _P, C.POINTER(StageStats)]),
-    "talaria_probe_copy": (C.c_int32, [_P, C.c_int32, _P, _P, C.c_int64, C.c_int32, _P]),
     "talaria_sync": (C.c_int32, [_P, _P]),
     "talaria_strerror": (C.c_char_p, [C.c_int32]),
     "talaria_last_cuda_error": (C.c_int32, [_P]),
@@ -451,11 +450,6 @@ class Talaria:
         plan = np.ascontiguousarray(plan, dtype=COPY_DTYPE)
         return int(lib().talaria_mark_dirty(_ptr(plan), plan.size, alloc_base, alloc_bytes, _ptr(staged_bitmap),
                                             _ptr(dirty_bitmap)))
-
-    def probe_copy(self, mechanism: int, src, dst, nbytes: int, ctas: int, stream=None):
-        """mechanism: 0 = 128-bit ld/st, 1 = 256-bit ld/st, 2 = TMA bulk copies."""
-        self._check(lib().talaria_probe_copy(self._h, mechanism, _ptr(src), _ptr(dst), nbytes, ctas,
-                                             _stream_ptr(stream)), "talaria_probe_copy")
 
     # -- completion and counters ---------------------------------------------
     def sync(self, stream=None):

@@ -4,6 +4,8 @@
 #include <cstring>
 #include <new>
 
+#include <cuda.h>   // types of the driver's pointer query only; the entry point is looked up at run time
+
 #include "internal.h"
 
 namespace tal {
@@ -102,6 +104,86 @@ talaria_status_t require_device_pointer(talaria_ctx *ctx, const void *p) {
     return TALARIA_OK;
   }
   return TALARIA_ERR_INVALID_ARG;
+}
+
+bool RangeCache::covers(uintptr_t p, uintptr_t bytes) const {
+  // last range that starts at or before p
+  auto it = std::upper_bound(v.begin(), v.end(), p, [](uintptr_t x, const AddrRange &r) { return x < r.lo; });
+  if (it == v.begin()) return false;
+  --it;
+  return p >= it->lo && p + bytes <= it->hi && p + bytes >= p;
+}
+
+void RangeCache::insert(AddrRange r) {
+  // whatever overlaps the new range described memory that has been freed since
+  v.erase(std::remove_if(v.begin(), v.end(), [&](const AddrRange &o) { return o.lo < r.hi && r.lo < o.hi; }), v.end());
+  v.insert(std::upper_bound(v.begin(), v.end(), r.lo, [](uintptr_t x, const AddrRange &o) { return x < o.lo; }), r);
+  if (v.size() > 4096) v.erase(v.begin(), v.begin() + 2048);   // bounded; dropped entries are simply asked again
+}
+
+// The allocation (or registration) that holds p, as the driver knows it.  The driver entry
+// point is resolved through the runtime, so the library does not link against libcuda.
+static bool query_allocation(const void *p, AddrRange *out) {
+  typedef CUresult (*pointer_attr_fn)(void *, CUpointer_attribute, CUdeviceptr);
+  static pointer_attr_fn fn = []() -> pointer_attr_fn {
+    void *f = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuPointerGetAttribute", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      (void)cudaGetLastError();
+      return nullptr;
+    }
+    return (pointer_attr_fn)f;
+  }();
+  if (!fn) return false;
+  CUdeviceptr start = 0;
+  size_t size = 0;
+  if (fn(&start, CU_POINTER_ATTRIBUTE_RANGE_START_ADDR, (CUdeviceptr)(uintptr_t)p) != CUDA_SUCCESS) return false;
+  if (fn(&size, CU_POINTER_ATTRIBUTE_RANGE_SIZE, (CUdeviceptr)(uintptr_t)p) != CUDA_SUCCESS) return false;
+  if (size == 0 || (uintptr_t)p < (uintptr_t)start || (uintptr_t)p >= (uintptr_t)start + size) return false;
+  *out = AddrRange{(uintptr_t)start, (uintptr_t)start + size};
+  return true;
+}
+
+talaria_status_t mapped_range(talaria_ctx *ctx, const void *host, int64_t bytes, void **dev_alias) {
+  if (bytes < 0) return TALARIA_ERR_INVALID_ARG;
+  const uintptr_t p = (uintptr_t)host, n = (uintptr_t)bytes;
+  // ranges registered through this context: their size is known exactly
+  for (const auto &r : ctx->registered) {
+    const uintptr_t lo = (uintptr_t)r.first, hi = lo + r.second;
+    if (p >= lo && p < hi) {
+      TAL_TRY(mapped_pointer(ctx, host, dev_alias));
+      return (!ctx->cfg.validate || p + n <= hi) ? TALARIA_OK : TALARIA_ERR_EXTENT;
+    }
+  }
+  TAL_TRY(mapped_pointer(ctx, host, dev_alias));
+  if (!ctx->cfg.validate || bytes <= 1) return TALARIA_OK;
+  if (p + n < p) return TALARIA_ERR_EXTENT;
+  if (ctx->host_ranges.covers(p, n)) return TALARIA_OK;
+  AddrRange a{};
+  if (query_allocation(host, &a)) {
+    ctx->host_ranges.insert(a);
+    return p + n <= a.hi ? TALARIA_OK : TALARIA_ERR_EXTENT;
+  }
+  // no range from the driver: at least the last byte must be pinned and mapped right behind the first
+  void *last = nullptr;
+  if (mapped_pointer(ctx, (const char *)host + (bytes - 1), &last) != TALARIA_OK) return TALARIA_ERR_EXTENT;
+  return ((uintptr_t)last - (uintptr_t)*dev_alias == n - 1) ? TALARIA_OK : TALARIA_ERR_EXTENT;
+}
+
+talaria_status_t require_device_range(talaria_ctx *ctx, const void *ptr, int64_t bytes) {
+  if (bytes < 0) return TALARIA_ERR_INVALID_ARG;
+  const uintptr_t p = (uintptr_t)ptr, n = (uintptr_t)bytes;
+  if (ctx->cfg.validate && p + n >= p && ctx->dev_ranges.covers(p, n ? n : 1)) return TALARIA_OK;
+  TAL_TRY(require_device_pointer(ctx, ptr));
+  if (!ctx->cfg.validate || bytes <= 1) return TALARIA_OK;
+  if (p + n < p) return TALARIA_ERR_EXTENT;
+  AddrRange a{};
+  if (query_allocation(ptr, &a)) {
+    ctx->dev_ranges.insert(a);
+    return p + n <= a.hi ? TALARIA_OK : TALARIA_ERR_EXTENT;
+  }
+  return require_device_pointer(ctx, (const char *)ptr + (bytes - 1)) == TALARIA_OK ? TALARIA_OK : TALARIA_ERR_EXTENT;
 }
 
 }  // namespace tal
@@ -231,6 +313,7 @@ extern "C" talaria_status_t talaria_host_unregister(talaria_ctx *ctx, void *host
     if (ctx->registered[k].first == (char *)host) {
       TAL_CUDA(ctx, cudaHostUnregister(host));
       ctx->registered.erase(ctx->registered.begin() + k);
+      ctx->host_ranges.v.clear();          // what the driver said about this memory no longer holds
       return TALARIA_OK;
     }
   }
@@ -243,9 +326,10 @@ extern "C" talaria_status_t talaria_sync(talaria_ctx *ctx, void *stream) {
   TAL_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
   // a copy kernel met a table entry outside the pool (possible only with validation off):
   // it skipped that chunk instead of touching foreign memory; report it once
-  if (const unsigned int word = *(volatile unsigned int *)ctx->status_host) {
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  if (*(volatile unsigned int *)ctx->status_host) {
     *(volatile unsigned int *)ctx->status_host = 0;
-    return (word & 2u) ? TALARIA_ERR_TIMEOUT : TALARIA_ERR_BAD_BLOCK_ID;
+    return TALARIA_ERR_BAD_BLOCK_ID;
   }
   return TALARIA_OK;
 }
@@ -260,7 +344,6 @@ extern "C" const char *talaria_strerror(talaria_status_t s) {
     case TALARIA_ERR_EXTENT: return "buffer smaller than the layout requires";
     case TALARIA_ERR_OVERLAP: return "stage plan ranges overlap";
     case TALARIA_ERR_CUDA: return "CUDA call failed (see talaria_last_cuda_error)";
-    case TALARIA_ERR_TIMEOUT: return "timeout";
     case TALARIA_ERR_NO_MEMORY: return "out of memory";
     default: return "unknown status";
   }

