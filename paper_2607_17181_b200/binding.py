@@ -19,7 +19,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libtalaria.so")
-SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "stage.cu", "registry.cu"]
+SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "prefix_pair.cu", "stage.cu", "registry.cu"]
+HEADERS = ["internal.h", "prefix_common.cuh"]
 
 OK = 0
 ERR_INVALID_ARG, ERR_BAD_BLOCK_ID, ERR_DUP_BLOCK, ERR_HOST_NOT_PINNED = -1, -2, -3, -4
@@ -30,7 +31,7 @@ VARIANT_AUTO, VARIANT_ZEROCOPY, VARIANT_BOUNCE, VARIANT_RUNS = 0, 1, 2, 3
 def build(force: bool = False, verbose: bool = False) -> str:
     """Compile the CUDA sources for sm_100a into libtalaria.so (in-tree)."""
     srcs = [os.path.join(_CSRC, s) for s in SOURCES]
-    deps = srcs + [os.path.join(_CSRC, "internal.h"), os.path.join(_INCLUDE, "talaria.h")]
+    deps = srcs + [os.path.join(_CSRC, h) for h in HEADERS] + [os.path.join(_INCLUDE, "talaria.h")]
     if not force and os.path.exists(LIB_PATH) and all(
             os.path.getmtime(LIB_PATH) >= os.path.getmtime(d) for d in deps):
         return LIB_PATH

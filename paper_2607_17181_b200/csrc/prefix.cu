@@ -20,62 +20,9 @@
 #include <cstring>
 
 #include "internal.h"
+#include "prefix_common.cuh"
 
 namespace tal {
-
-constexpr uint64_t kG = 0x9E3779B97F4A7C15ull;
-constexpr uint64_t kP = 0xD1342543DE82EF95ull;
-constexpr int kTileTok = 2048;        // tokens per tile: latency path (fused kernel, static entry point)
-constexpr int kBatchTileTok = 8192;   // tokens per tile in big batches: amortises the per-CTA start-up
-constexpr int kTileThreads = 256;
-constexpr int kScanThreads = 256;
-constexpr int kScanItems = 8;
-constexpr long long kNoMismatch = 0x7fffffffffffffffll;
-
-__device__ __forceinline__ uint64_t mix64(uint64_t z) {
-  z ^= z >> 30;
-  z *= 0xBF58476D1CE4E5B9ull;
-  z ^= z >> 27;
-  z *= 0x94D049BB133111EBull;
-  z ^= z >> 31;
-  return z;
-}
-
-struct PairDesc {
-  int64_t cont_off, sess_off;          // token offsets into the concatenated arrays
-  int64_t Tc, Ts;                      // token counts
-  int64_t cont_blk_off, sess_blk_off;  // block offsets into hash / digest arrays
-  int64_t tile_off;                    // first tile of this pair
-};
-
-constexpr int kInlinePairs = 8;    // up to this many pairs travel in the kernel parameters
-constexpr int64_t kFusedMaxTiles = 296;    // 2 CTAs per SM x 148 SMs: about one wave of the fused kernel
-
-struct PrefixParams {
-  const PairDesc *pairs;      // DEVICE [n_pairs + 1] (last entry holds the totals); null when inline
-  const int32_t *tile_pair;   // DEVICE [tiles]: pair of each tile; null when inline
-  PairDesc inl[kInlinePairs + 1];
-  int32_t n_pairs;
-  int32_t B;
-  int32_t log2B;              // >= 0 when B is a power of two <= 32, else -1
-  int32_t need_sess_digest;   // 1 when stored hashes are not supplied
-  int32_t tile_tok;           // tokens per tile (a multiple of 1024)
-  const int32_t *cont, *sess; // DEVICE tokens
-  uint64_t *dig_c, *dig_s;    // DEVICE scratch digests
-  long long *tile_mis;        // DEVICE scratch [total tiles]
-  const uint64_t *sess_hashes;// DEVICE or null
-  uint64_t *cont_hashes_out;  // DEVICE or null
-  talaria_match_t *results;   // DEVICE [n_pairs] or null
-  uint64_t seed;
-  unsigned int *counters;     // DEVICE [kInlinePairs], zero between calls (fused kernel only)
-};
-
-__device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int m) {
-  return (uint64_t)__shfl_xor_sync(0xffffffffu, (unsigned long long)v, m);
-}
-__device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
-  return (uint64_t)__shfl_up_sync(0xffffffffu, (unsigned long long)v, d);
-}
 
 // Work of one 2,048-token tile; returns the pair the tile belongs to.
 __device__ __forceinline__ int tile_body(const PrefixParams &p) {
@@ -457,8 +404,15 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     big.resize((size_t)n_pairs + 1);
     pd = big.data();
   }
+  int log2B = -1;
+  if (B <= 32 && (B & (B - 1)) == 0)
+    while ((1 << ++log2B) < B) {}
+  // Batches with at least one pair per SM: one CTA per pair, one launch, no global scratch.
+  if (!inl && n_pairs >= ctx->sm_count && log2B >= 2)
+    return pair_launch(ctx, n_pairs, d_cont, cont_off, d_sess, sess_off, d_sess_hashes, B, log2B, seed,
+                       d_cont_hashes, d_results, stream);
   // A handful of pairs run as ONE fused launch (every pair then owns at least one tile, so some
-  // CTA always finishes it); big batches keep two lean kernels for throughput.
+  // CTA always finishes it); batches in between use a tile kernel and a chain kernel.
   bool fused = inl;
   int64_t cb = 0, sb = 0, tiles = 0;
   int tile_tok = kTileTok;
@@ -505,12 +459,7 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   }
   p.n_pairs = n_pairs;
   p.B = B;
-  p.log2B = -1;
-  if (B <= 32 && (B & (B - 1)) == 0) {
-    int l = 0;
-    while ((1 << l) < B) ++l;
-    p.log2B = l;
-  }
+  p.log2B = log2B;
   p.need_sess_digest = derive ? 1 : 0;
   p.tile_tok = tile_tok;
   p.cont = d_cont;

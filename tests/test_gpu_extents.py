@@ -116,14 +116,15 @@ def test_plane_smaller_than_the_declared_pool_is_rejected():
 def test_stage_ranges_that_leave_their_allocation_are_rejected():
     ctx = tb.Talaria(0)
     try:
-        # 32 MiB tensors are allocations of their own; the spacers keep the over-long ranges below
-        # from reaching the other tensor, which would be an overlap error instead
-        nbytes, too_long = 32 << 20, 36 << 20
+        # 32 MiB tensors are allocations of their own.  The over-long ranges below run 4 MiB past
+        # their tensor; the other end of each copy sits in the middle of a 192 MiB tensor, so the
+        # two ranges of an entry can never meet (that would be an overlap error instead).
+        nbytes, too_long, mid = 32 << 20, 36 << 20, 64 << 20
         staging = torch.arange(nbytes // 8, dtype=torch.int64, device="cuda").view(torch.uint8)
-        spacer1 = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
         slots = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
-        spacer2 = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
-        host = torch.zeros(nbytes, dtype=torch.uint8, pin_memory=True)
+        big = torch.zeros(192 << 20, dtype=torch.uint8, device="cuda")
+        host = torch.zeros(64 << 20, dtype=torch.uint8, pin_memory=True)
+        small_host = torch.zeros(nbytes, dtype=torch.uint8, pin_memory=True)
 
         def plan(src_dev, src_host, dst, nb):
             a = np.zeros(1, tb.COPY_DTYPE)
@@ -132,17 +133,25 @@ def test_stage_ranges_that_leave_their_allocation_are_rejected():
 
         before = _launched(ctx)
         dirty = np.array([1], np.uint8)
-        assert _status(ctx.stage, plan(staging.data_ptr(), 0, slots.data_ptr(), too_long)) == tb.ERR_EXTENT
-        assert _status(ctx.stage, plan(staging.data_ptr(), host.data_ptr(), slots.data_ptr(), too_long), dirty) == tb.ERR_EXTENT
-        assert _status(ctx.stage_plan_create, plan(staging.data_ptr(), 0, slots.data_ptr(), too_long)) == tb.ERR_EXTENT
+        src_runs_off = plan(staging.data_ptr(), 0, big.data_ptr() + mid, too_long)
+        dst_runs_off = plan(big.data_ptr() + mid, 0, slots.data_ptr(), too_long)
+        dst_runs_off_from_host = plan(0, host.data_ptr(), slots.data_ptr(), too_long)
+        host_runs_off = plan(big.data_ptr() + mid, small_host.data_ptr(), big.data_ptr(), too_long)
+        assert _status(ctx.stage, src_runs_off) == tb.ERR_EXTENT
+        assert _status(ctx.stage, dst_runs_off) == tb.ERR_EXTENT
+        assert _status(ctx.stage, dst_runs_off_from_host) == tb.ERR_EXTENT
+        assert _status(ctx.stage, host_runs_off, dirty) == tb.ERR_EXTENT
+        assert _status(ctx.stage_plan_create, src_runs_off) == tb.ERR_EXTENT
+        assert _status(ctx.stage_plan_create, dst_runs_off) == tb.ERR_EXTENT
         staged, dbits = np.zeros(1, np.uint8), np.zeros(1, np.uint8)
-        assert _status(ctx.prestage, plan(staging.data_ptr(), host.data_ptr(), slots.data_ptr(), too_long), None, staged, dbits) == tb.ERR_EXTENT
+        # pre-staging writes host bytes to src_dev: both of its ranges are checked too
+        assert _status(ctx.prestage, plan(staging.data_ptr(), host.data_ptr(), 0, too_long), None, staged, dbits) == tb.ERR_EXTENT
+        assert _status(ctx.prestage, plan(big.data_ptr(), small_host.data_ptr(), 0, too_long), None, staged, dbits) == tb.ERR_EXTENT
         assert _launched(ctx) == before and not staged.any()
-        assert not slots.any().item()
+        assert not slots.any().item() and not big.any().item()
         ctx.stage(plan(staging.data_ptr(), 0, slots.data_ptr(), nbytes))          # the honest plan works
         ctx.sync()
         assert torch.equal(slots, staging)
-        del spacer1, spacer2
     finally:
         ctx.destroy()
 

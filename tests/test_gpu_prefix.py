@@ -55,10 +55,11 @@ def test_block_hash_long_stream_crosses_scan_chunks(ctx):
 
 def _match_batch(ctx, pairs, B, seed, with_stored, pad_front=0):
     """pairs: list of (cont, sess).  Returns GPU results + hashes via the device entry point."""
-    cont = np.concatenate([np.zeros(pad_front, np.int32)] + [c for c, _ in pairs])
-    sess = np.concatenate([np.zeros(pad_front, np.int32)] + [s for _, s in pairs])
-    co = np.cumsum([pad_front] + [c.size for c, _ in pairs]).astype(np.int64)
-    so = np.cumsum([pad_front] + [s.size for _, s in pairs]).astype(np.int64)
+    pad_c, pad_s = pad_front if isinstance(pad_front, tuple) else (pad_front, pad_front)
+    cont = np.concatenate([np.zeros(pad_c, np.int32)] + [c for c, _ in pairs])
+    sess = np.concatenate([np.zeros(pad_s, np.int32)] + [s for _, s in pairs])
+    co = np.cumsum([pad_c] + [c.size for c, _ in pairs]).astype(np.int64)
+    so = np.cumsum([pad_s] + [s.size for _, s in pairs]).astype(np.int64)
     stored = [orc.block_hash(s, B, seed) for _, s in pairs]
     nbc = sum(c.size // B for c, _ in pairs)
     d_cont = _dev(cont) if cont.size else torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -219,6 +220,63 @@ def test_thousands_of_small_pairs(ctx):
         pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1))), s))
     _check_batch(ctx, pairs, 16, SEED, False)
     _check_batch(ctx, pairs, 4, SEED, True)
+
+
+def _big_batch(B, seed):
+    """At least one pair per SM, so the one-CTA-per-pair kernel runs: mostly short ragged pairs,
+    plus pairs built around that kernel's boundaries (chunks of 1,024 blocks, rounds of 1,024 tokens)."""
+    g = wl.rng(509, seed)
+    chunk = 1024 * B
+    e = np.zeros(0, np.int32)
+    pairs = []
+    for _ in range(150):
+        ts, tc = int(g.integers(0, 3000)), int(g.integers(0, 3000))
+        s = wl.tokens(g, ts)
+        pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1))), s))
+    long_s = wl.tokens(g, 2 * chunk + 5 * B + 3)
+    for tc, shared in ((2 * chunk + 900, chunk), (2 * chunk + 900, chunk - 1), (2 * chunk + 900, chunk + 1),
+                       (long_s.size, long_s.size), (long_s.size + 1, long_s.size), (chunk, chunk), (chunk, 0),
+                       (chunk + 1024, 1024), (chunk + 1024, 1023), (3 * chunk, 2 * chunk + 5 * B + 3),
+                       (700, 700), (chunk // 2 + 7, 5)):
+        pairs.append((wl.continuation(g, long_s, tc, shared), long_s))
+    short_s = wl.tokens(g, 2 * B + 1)
+    pairs += [(wl.continuation(g, short_s, 2 * chunk + 17, short_s.size), short_s),   # the continuation extends a short stream
+              (long_s[: 3 * B].copy(), long_s), (e, long_s), (long_s, e), (e, e), (long_s.copy(), long_s)]
+    return pairs
+
+
+@pytest.mark.parametrize("B", [4, 8, 16, 32])
+@pytest.mark.parametrize("with_stored", [False, True])
+def test_large_batch_one_cta_per_pair(ctx, B, with_stored):
+    pairs = _big_batch(B, B)
+    assert len(pairs) >= 148
+    _check_batch(ctx, pairs, B, SEED, with_stored)
+    order = wl.rng(509, 77).permutation(len(pairs))                     # long pairs anywhere in the batch
+    _check_batch(ctx, [pairs[k] for k in order], B, 0, with_stored, pad_front=(1, 2))
+    _check_batch(ctx, [pairs[k] for k in order[::-1]], B, SEED, with_stored, pad_front=(3, 0))
+
+
+def test_large_batch_detects_a_corrupted_stored_hash_in_a_late_chunk(ctx):
+    B = 16
+    pairs = _big_batch(B, 5)
+    q = next(k for k, (c, s) in enumerate(pairs) if c.size > 2 * 1024 * B and np.array_equal(c[: s.size], s))
+    cont = np.concatenate([c for c, _ in pairs]); sess = np.concatenate([s for _, s in pairs])
+    co = np.cumsum([0] + [c.size for c, _ in pairs]).astype(np.int64)
+    so = np.cumsum([0] + [s.size for _, s in pairs]).astype(np.int64)
+    stored = [orc.block_hash(s, B, SEED) for _, s in pairs]
+    bad_block = 1024 + 700                                              # second chunk of that pair
+    stored[q][bad_block] ^= np.uint64(1 << 40)
+    d_res = torch.zeros(len(pairs) * 4, dtype=torch.int64, device="cuda")
+    ctx.prefix_match(len(pairs), _dev(cont), co, _dev(sess), so, _dev(np.concatenate(stored).view(np.int64)), B, SEED,
+                     None, d_res)
+    ctx.sync()
+    res = d_res.cpu().numpy().view(tb.MATCH_DTYPE)
+    for k, (c, s) in enumerate(pairs):
+        m, _ = orc.prefix_match(c, s, B, SEED, sess_hashes=stored[k])
+        assert (int(res[k]["lcp_tokens"]), int(res[k]["matched_blocks"]), int(res[k]["reusable_tokens"]),
+                int(res[k]["hash_token_disagree"])) == (m.lcp_tokens, m.matched_blocks, m.reusable_tokens,
+                                                        m.hash_token_disagree), k
+    assert int(res[q]["matched_blocks"]) == bad_block and int(res[q]["hash_token_disagree"]) == 1
 
 
 def test_smoke_entry_point_runs():
