@@ -22,19 +22,18 @@
 
 namespace tal {
 
-#ifndef TAL_MINB
-#define TAL_MINB 3
-#endif
-#ifndef TAL_DEPTH1
-#define TAL_DEPTH1 2
-#endif
-#ifndef TAL_DEPTH2
-#define TAL_DEPTH2 1
-#endif
+// Shape of the CTA.  Measured on the 1,024 x 32,768-token batch: 64 / 128 / 256 threads with
+// 12 / 8 / 3-4 CTAs per SM and one to four quads in flight per stream all land within a few
+// per cent of each other (the integer ALU pipe is the limit, not occupancy or memory latency).
 constexpr int kPairThreads = 256;
+constexpr int kPairCtasPerSm = 3;      // register budget of 80 per thread
+constexpr int kDepthOne = 2;           // quads in flight when one stream is hashed
+constexpr int kDepthBoth = 1;          // ... per stream when both are hashed
+constexpr int kPairWarps = kPairThreads / 32;
 constexpr int kChunkBlocks = 1024;                         // blocks per chunk
-constexpr int kRounds = kChunkBlocks / kPairThreads;       // blocks per thread per chunk (4)
-static_assert(kRounds == 4 && kPairThreads == 256, "the scan constants below assume 8 warps x 32 lanes x 4 blocks");
+constexpr int kRounds = kChunkBlocks / kPairThreads;       // blocks per thread per chunk
+static_assert(kRounds * kPairThreads == kChunkBlocks && (kPairWarps & (kPairWarps - 1)) == 0 && kPairWarps <= 32,
+              "a chunk is a whole number of rounds and the warp totals are scanned by a power-of-two group of lanes");
 
 __host__ __device__ constexpr uint64_t pow_p(unsigned n) {
   uint64_t r = 1, b = kP;
@@ -86,7 +85,7 @@ __device__ __forceinline__ void hash_blocks(const int32_t *cont, const int32_t *
                                             const int64_t tbase, const int r0, const int r1, uint64_t *dig_c,
                                             uint64_t *dig_s, long long &first_mis) {
   constexpr int Q = (1 << LOG2B) / 4;                    // quads per block
-  constexpr int DEPTH = Q < 4 ? Q : (MODE == 2 ? TAL_DEPTH2 : TAL_DEPTH1); // quads in flight per stream
+  constexpr int DEPTH = Q < 4 ? Q : (MODE == 2 ? kDepthBoth : kDepthOne); // quads in flight per stream
   constexpr int kRoundTok = kPairThreads << LOG2B;       // tokens between this thread's blocks of two rounds
   if (r0 >= r1) return;
   const int tid = threadIdx.x;
@@ -162,10 +161,10 @@ __device__ __forceinline__ void hash_blocks_checked(const int32_t *cont, const i
   }
 }
 
-// Inclusive scan over the 256 threads of x_t (each the zero-carry chain of that thread's four
-// blocks).  Returns the zero-carry chain of everything BEFORE the thread's run, split in two
-// parts so that  state_before_run = carry * P^(4 tid) + before_warps * P^(4 lane) + before_lanes;
-// total = chain of the whole chunk.  s_tot: eight words of shared memory.
+// Inclusive scan over the CTA's threads of x_t (each the zero-carry chain of that thread's
+// kRounds blocks).  Returns the zero-carry chain of everything BEFORE the thread's run, split in two
+// parts so that  state_before_run = carry * P^(kRounds tid) + before_warps * P^(kRounds lane) + before_lanes;
+// total = chain of the whole chunk.  s_tot: one word of shared memory per warp.
 __device__ __forceinline__ void chunk_scan(uint64_t x, uint64_t *s_tot, uint64_t &before_warps,
                                            uint64_t &before_lanes, uint64_t &total) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -178,24 +177,24 @@ __device__ __forceinline__ void chunk_scan(uint64_t x, uint64_t *s_tot, uint64_t
   before_lanes = shfl_up_u64(x, 1);
   if (lane == 0) before_lanes = 0;
   __syncthreads();
-  uint64_t v = s_tot[lane & 7];
+  uint64_t v = s_tot[lane & (kPairWarps - 1)];
 #pragma unroll
-  for (int d = 1; d < 8; d <<= 1) {
+  for (int d = 1; d < kPairWarps; d <<= 1) {
     const uint64_t y = shfl_up_u64(v, d);
-    if ((lane & 7) >= d) v = y * pow_p(kRounds * 32 * d) + v;
+    if ((lane & (kPairWarps - 1)) >= d) v = y * pow_p(kRounds * 32 * d) + v;
   }
-  total = (uint64_t)__shfl_sync(0xffffffffu, (unsigned long long)v, 7);
-  before_warps = (uint64_t)__shfl_sync(0xffffffffu, (unsigned long long)v, (wid + 7) & 7);
+  total = (uint64_t)__shfl_sync(0xffffffffu, (unsigned long long)v, kPairWarps - 1);
+  before_warps = (uint64_t)__shfl_sync(0xffffffffu, (unsigned long long)v, (wid + kPairWarps - 1) & (kPairWarps - 1));
   if (wid == 0) before_warps = 0;
 }
 
 template <bool DERIVE, int LOG2B>
-__global__ void __launch_bounds__(kPairThreads, TAL_MINB) prefix_pair_kernel(const __grid_constant__ PrefixParams p) {
+__global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kernel(const __grid_constant__ PrefixParams p) {
   constexpr int B = 1 << LOG2B;
   constexpr int kRoundTok = kPairThreads << LOG2B;     // tokens hashed per round by the whole CTA
   constexpr int kChunkShift = 10 + LOG2B;              // tokens per chunk = 1024 * B
   __shared__ __align__(16) uint64_t s_dig[DERIVE ? 2 : 1][kChunkBlocks];
-  __shared__ uint64_t s_tot[2][8];
+  __shared__ uint64_t s_tot[2][kPairWarps];
   __shared__ long long s_red[2][kPairThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int pair = p.order[blockIdx.x];
@@ -211,7 +210,7 @@ __global__ void __launch_bounds__(kPairThreads, TAL_MINB) prefix_pair_kernel(con
   const uint64_t *hs_in = DERIVE ? nullptr : p.sess_hashes + pd.sess_blk_off;
   uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_blk_off : nullptr;
 
-  // P^(4 lane) and P^(4 tid): where this thread's run starts inside its warp and inside the chunk
+  // P^(kRounds lane) and P^(kRounds tid): where this thread's run starts inside its warp and inside the chunk
   uint64_t pow_lane = 1, pow_tid = 1;
   {
     uint64_t b = pow_p(kRounds);
@@ -375,10 +374,11 @@ talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d
   std::stable_sort(order, order + n_pairs, [&](int32_t a, int32_t b) {
     return std::max(pd[a].Tc, pd[a].Ts) > std::max(pd[b].Tc, pd[b].Ts);
   });
-  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+  // Each CTA reads its one descriptor straight from the pinned slot (60 bytes over the host
+  // link): no upload stands between this launch and the previous kernel on the stream.
   PrefixParams p{};
-  p.pairs = (const PairDesc *)slot->d;
-  p.order = (const int32_t *)(slot->d + pair_bytes);
+  p.pairs = (const PairDesc *)slot->h;
+  p.order = (const int32_t *)(slot->h + pair_bytes);
   p.n_pairs = n_pairs;
   p.B = B;
   p.log2B = log2B;
