@@ -78,6 +78,8 @@ typedef struct {
   int32_t validate;       /* 0 = skip host-side table / plan validation; default 1            */
   int32_t zc_ctas;        /* grid size of zero-copy kernels; 0 = built-in (leaves SMs free)   */
   int32_t pack_ctas;      /* grid size of the bounce variant's pack / unpack kernels; 0 = 64  */
+  int64_t host_match_bytes; /* staging (pinned + device, allocated once at create) of            */
+                            /* talaria_prefix_match_host; 0 = 16 MiB, at least 1 MiB             */
 } talaria_config_t;
 
 /* Device-side paged KV pool (Sec. 4.3; descriptor fields of App. C "Attention-layout
@@ -183,9 +185,13 @@ talaria_status_t talaria_prefix_match(talaria_ctx *ctx, int32_t n_pairs,
                                       uint64_t seed, uint64_t *d_cont_hashes_out,
                                       talaria_match_t *d_results, void *stream);
 
-/* Same computation with every array in HOST memory (pageable or pinned): tokens
- * are copied to the device, matched by the same kernels, and results / hashes are
- * copied back.  Synchronous: returns after the results are in host memory. */
+/* Same computation with every array in HOST memory (pageable or pinned).  The inputs are
+ * gathered into the context's pinned staging buffer, go to the device in ONE copy, are
+ * matched by the same kernels, and hashes and results come back in ONE copy.  Nothing is
+ * allocated or freed: staging was sized at talaria_create (host_match_bytes).  A batch
+ * larger than the staging is processed as several sub-batches of whole pairs; a single
+ * pair that does not fit is TALARIA_ERR_EXTENT.  Synchronous: returns after the results
+ * are in host memory. */
 talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
                                            const int32_t *h_cont_tokens, const int64_t *cont_offsets,
                                            const int32_t *h_sess_tokens, const int64_t *sess_offsets,
@@ -316,8 +322,12 @@ talaria_status_t talaria_kv_restore_pages(talaria_ctx *ctx, const talaria_kv_lay
                                           int64_t n_blocks, const void *host_pool, int64_t pool_bytes,
                                           const int64_t *page_offsets, void *stream);
 
-/* Several sessions in one call: each transfer is enqueued in turn on `stream`; restore tables
- * are checked against each other first (no block may be claimed twice). */
+/* Several sessions in one call.  Every argument of every session is checked before anything is
+ * enqueued; restore tables are also checked against each other (no block may be claimed
+ * twice).  Sessions small enough for the zero-copy kernel whose images share their layer and
+ * plane strides (any page-first images; layer-first images of equal block count) are moved by
+ * ONE fused launch; with at most 256 blocks in total even its descriptor travels in the kernel
+ * parameters.  Larger sessions use the copy-engine variants, one after the other on `stream`. */
 typedef struct {
   const int32_t *block_table; /* HOST */
   int64_t first_block, n_blocks;

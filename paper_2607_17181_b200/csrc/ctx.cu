@@ -202,6 +202,12 @@ static void destroy_impl(talaria_ctx *ctx) {
     if (ln.fork) cudaEventDestroy(ln.fork);
     if (ln.buf) cudaFree(ln.buf);
   }
+  if (ctx->reload_stream) {
+    cudaStreamSynchronize(ctx->reload_stream);
+    cudaStreamDestroy(ctx->reload_stream);
+  }
+  if (ctx->reload_fork) cudaEventDestroy(ctx->reload_fork);
+  if (ctx->reload_done) cudaEventDestroy(ctx->reload_done);
   for (auto &s : ctx->ring) {
     if (s.used) cudaEventSynchronize(s.ev);
     if (s.ev) cudaEventDestroy(s.ev);
@@ -214,6 +220,7 @@ static void destroy_impl(talaria_ctx *ctx) {
   if (ctx->status_host) cudaFreeHost(ctx->status_host);
   if (ctx->prefix_scratch.p) cudaFree(ctx->prefix_scratch.p);
   if (ctx->host_tok.p) cudaFree(ctx->host_tok.p);
+  if (ctx->match_pin) cudaFreeHost(ctx->match_pin);
   for (auto &r : ctx->registered) cudaHostUnregister(r.first);
   (void)cudaGetLastError();
   delete ctx;
@@ -234,6 +241,8 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
   if (!cfg) ctx->cfg.validate = 1;
   if (ctx->cfg.bounce_bytes <= 0) ctx->cfg.bounce_bytes = 128ll << 20;
   if (ctx->cfg.bounce_bytes < (1 << 20)) ctx->cfg.bounce_bytes = 1 << 20;
+  if (ctx->cfg.host_match_bytes <= 0) ctx->cfg.host_match_bytes = 16ll << 20;
+  if (ctx->cfg.host_match_bytes < (1 << 20)) ctx->cfg.host_match_bytes = 1 << 20;
   if (const char *v = getenv("TALARIA_VARIANT")) {
     int x = atoi(v);
     if (x >= TALARIA_VARIANT_AUTO && x <= TALARIA_VARIANT_RUNS) ctx->cfg.variant = x;
@@ -260,11 +269,16 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
     TAL_CUDA(ctx, cudaMalloc((void **)&ctx->prefix_counters, 64 * sizeof(unsigned int)));
     TAL_CUDA(ctx, cudaMemset(ctx->prefix_counters, 0, 64 * sizeof(unsigned int)));
     TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->prefix_done, cudaEventDisableTiming));
+    TAL_TRY(grow(ctx, &ctx->host_tok, (size_t)ctx->cfg.host_match_bytes));
+    TAL_CUDA(ctx, cudaHostAlloc((void **)&ctx->match_pin, ctx->host_tok.cap, cudaHostAllocDefault));
     // Internal streams run at the highest priority: their kernels are short packing
     // steps that gate copy-engine transfers, so they should not queue behind a long
     // kernel of the caller's (for example a staging copy on another stream).
     int prio_least = 0, prio_greatest = 0;
     TAL_CUDA(ctx, cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+    TAL_CUDA(ctx, cudaStreamCreateWithPriority(&ctx->reload_stream, cudaStreamNonBlocking, prio_least));
+    TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->reload_fork, cudaEventDisableTiming));
+    TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->reload_done, cudaEventDisableTiming));
     for (auto &ln : ctx->lane) {
       for (int j = 0; j < 2; ++j) {
         TAL_CUDA(ctx, cudaStreamCreateWithPriority(&ln.s[j], cudaStreamNonBlocking, prio_greatest));

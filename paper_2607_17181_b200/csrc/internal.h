@@ -13,6 +13,7 @@ namespace tal {
 constexpr int kRing = 8;              // descriptor slots in flight
 constexpr size_t kSlotBytes = 2u << 20;  // initial size of each slot (pinned + device)
 constexpr int kLanes = 2;             // 0: offload (device->host), 1: restore (host->device)
+constexpr int64_t kReloadPiece = 32ll << 20;   // largest single host->device copy of a weight reload
 
 struct DescSlot {
   char *h = nullptr;                  // pinned staging
@@ -57,12 +58,18 @@ struct talaria_ctx {
   tal::DescSlot ring[tal::kRing];
   int ring_next = 0;
   tal::BounceLane lane[tal::kLanes];
+  // Host-sourced reloads of a staged switch run on a stream of their own, cut into bounded
+  // pieces, so a KV restore issued meanwhile gets its turns on the host link (Sec. 3.4 charges
+  // the restore, not the weight reload, to the admission budget).
+  cudaStream_t reload_stream = nullptr;
+  cudaEvent_t reload_fork = nullptr, reload_done = nullptr;
   tal::DevBuf prefix_scratch;         // digests + per-tile mismatch positions
   unsigned int *prefix_counters = nullptr;  // per-pair tile counters of the fused prefix kernel (zero at rest)
   cudaEvent_t prefix_done = nullptr;  // end of the last prefix call (its scratch is shared)
   bool prefix_busy = false;
   cudaStream_t prefix_stream = nullptr;  // stream of that call (same stream: already ordered)
-  tal::DevBuf host_tok;               // device copies for talaria_prefix_match_host
+  tal::DevBuf host_tok;               // device side of talaria_prefix_match_host's staging (fixed size)
+  char *match_pin = nullptr;          // pinned side, same size and layout
   std::vector<std::pair<char *, size_t>> registered;
   tal::RangeCache host_ranges;        // pinned host allocations seen so far
   tal::RangeCache dev_ranges;         // device allocations seen so far

@@ -52,7 +52,7 @@ __device__ __forceinline__ void decode_chunk(const KvCopyParams &p, int64_t w, i
 // TO_IMAGE: pool -> image (offload / gather); else image -> pool (restore / scatter).
 // VB: bytes per access (16 or 32); every lane keeps 128 bytes in flight per step.
 template <bool TO_IMAGE, int VB>
-__global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant__ KvCopyParams p) {
+__device__ __forceinline__ void kv_copy_vec_body(const KvCopyParams &p) {
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -93,6 +93,33 @@ __global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant_
       for (int k = lane; k < n16; k += 32) __stcs((int4 *)dst + k, __ldcs((const int4 *)src + k));
     }
   }
+}
+
+template <bool TO_IMAGE, int VB>
+__global__ void __launch_bounds__(512) kv_copy_vec_kernel(const __grid_constant__ KvCopyParams p) {
+  kv_copy_vec_body<TO_IMAGE, VB>(p);
+}
+
+// Transfers of a few blocks carry their whole descriptor in the kernel parameters: plane
+// addresses, table slice and (for page slabs or fused sessions) per-block offsets.  Nothing is
+// uploaded and no descriptor slot is taken, which is most of the fixed cost of a small copy.
+constexpr int kInlinePlanes = 256;
+constexpr int kInlineBlocks = 256;
+struct KvCopyInline {
+  KvCopyParams p;                       // plane_base / table / page_off are filled in by the kernel
+  const void *planes[kInlinePlanes];
+  int64_t page_off[kInlineBlocks];
+  int32_t table[kInlineBlocks];
+  int32_t has_page_off;
+};
+
+template <bool TO_IMAGE, int VB>
+__global__ void __launch_bounds__(512) kv_copy_vec_inline_kernel(const __grid_constant__ KvCopyInline q) {
+  KvCopyParams p = q.p;
+  p.plane_base = q.planes;
+  p.table = q.table;
+  p.page_off = q.has_page_off ? q.page_off : nullptr;
+  kv_copy_vec_body<TO_IMAGE, VB>(p);
 }
 
 // Any chunk size / alignment: plain byte copies (odd shapes only).
@@ -255,6 +282,41 @@ static talaria_status_t launch_copy(talaria_ctx *ctx, const KvCopyParams &p, int
   return TALARIA_OK;
 }
 
+// The same launch with the descriptor in the kernel parameters.  planes: L*P device addresses (host
+// array); table: n ids; page_off: n offsets or null.  Needs vec != 0 and the inline limits.
+static talaria_status_t launch_inline(talaria_ctx *ctx, bool to_image, const KvCopyParams &p, int vec,
+                                      int64_t grid_cap, const void *const *planes, int64_t n_planes,
+                                      const int32_t *table, const int64_t *page_off, int64_t n,
+                                      cudaStream_t stream) {
+  if (p.w1 <= p.w0) return TALARIA_OK;
+  KvCopyInline q{};
+  q.p = p;
+  memcpy(q.planes, planes, (size_t)n_planes * sizeof(void *));
+  memcpy(q.table, table, (size_t)n * sizeof(int32_t));
+  if (page_off) memcpy(q.page_off, page_off, (size_t)n * sizeof(int64_t));
+  q.has_page_off = page_off ? 1 : 0;
+  if ((uintptr_t)p.img % 32 != 0 && vec == 32) vec = 16;
+  const int threads = 512;
+  const int64_t parts = (p.chunk_bytes + kPart - 1) / kPart;
+  const int64_t warps = (p.w1 - p.w0) * parts;
+  const int64_t need = (warps + threads / 32 - 1) / (threads / 32);
+  const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(need, grid_cap));
+  if (to_image) {
+    if (vec == 32) kv_copy_vec_inline_kernel<true, 32><<<grid, threads, 0, stream>>>(q);
+    else           kv_copy_vec_inline_kernel<true, 16><<<grid, threads, 0, stream>>>(q);
+  } else {
+    if (vec == 32) kv_copy_vec_inline_kernel<false, 32><<<grid, threads, 0, stream>>>(q);
+    else           kv_copy_vec_inline_kernel<false, 16><<<grid, threads, 0, stream>>>(q);
+  }
+  TAL_CUDA(ctx, cudaGetLastError());
+  ctx->counters.kernel_launches++;
+  return TALARIA_OK;
+}
+
+static bool fits_inline(int64_t n_planes, int64_t n, int vec, const void *img) {
+  return n_planes <= kInlinePlanes && n <= kInlineBlocks && vec != 0 && (uintptr_t)img % 16 == 0;
+}
+
 static talaria_status_t launch_dir(talaria_ctx *ctx, bool to_image, const KvCopyParams &p, int vec,
                                    int64_t grid_cap, cudaStream_t stream) {
   return to_image ? launch_copy<true>(ctx, p, vec, grid_cap, stream)
@@ -284,6 +346,28 @@ static int64_t count_id_runs(const int32_t *bt, int64_t n) {
   return runs;
 }
 
+// How a host-side transfer crosses the link (the measured crossover: profiles/crossover table).
+static int choose_variant(const talaria_ctx *ctx, const Plan &pl, const talaria_host_layout_t *hl,
+                          const int32_t *bt, int64_t n, bool to_image) {
+  const BounceLane &ln = ctx->lane[to_image ? 0 : 1];
+  const int64_t payload = pl.chunks * pl.C;
+  const int64_t dma_min = ctx->cfg.dma_min_bytes > 0 ? ctx->cfg.dma_min_bytes : (8ll << 20);
+  const int64_t seg_bytes = pl.run_chunks * pl.C;
+  const bool bounce_ok = (int64_t)ln.half >= pl.C;
+  int variant = ctx->cfg.variant;
+  if (variant == TALARIA_VARIANT_AUTO) {
+    variant = TALARIA_VARIANT_ZEROCOPY;
+    if (bounce_ok && payload >= dma_min && seg_bytes >= (256 << 10)) variant = TALARIA_VARIANT_BOUNCE;
+    // a table of few long runs of adjacent ids needs no kernel at all
+    if (payload >= dma_min && (hl->stride_block == pl.C || n == 1)) {
+      const int64_t copies = pl.L * pl.P * count_id_runs(bt, n);
+      if (copies <= 1024 && payload / copies >= (1 << 20)) variant = TALARIA_VARIANT_RUNS;
+    }
+  }
+  if (variant == TALARIA_VARIANT_BOUNCE && !bounce_ok) variant = TALARIA_VARIANT_ZEROCOPY;
+  return variant;
+}
+
 // to_image: offload / gather; img_on_device: the image is device memory (gather / scatter).
 static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const int32_t *table,
                                     int64_t first, int64_t n, void *img, const talaria_host_layout_t *hl,
@@ -305,59 +389,47 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
     if (((uintptr_t)img_dev) % 16 != 0) pl.vec = 0;
   }
 
-  // descriptor: plane pointers, then the table slice
-  const size_t ptr_bytes = (size_t)(pl.L * pl.P) * sizeof(void *);
-  const size_t desc_bytes = ptr_bytes + (size_t)n * sizeof(int32_t);
-  DescSlot *slot;
-  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
-  memcpy(slot->h, kv->plane_base, ptr_bytes);
-  memcpy(slot->h + ptr_bytes, bt, (size_t)n * sizeof(int32_t));
-  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
-
   KvCopyParams p{};
   p.num_blocks = kv->num_blocks;
   p.status = ctx->status_dev;
-  p.plane_base = (const void *const *)slot->d;
-  p.table = (const int32_t *)(slot->d + ptr_bytes);
   p.chunk_bytes = pl.C;
   p.ord = pl.ord;
-
   const int64_t payload = pl.chunks * pl.C;
   ctx->counters.payload_bytes += payload;
 
-  if (img_on_device) {
-    p.img = (char *)img_dev;
-    set_image_strides(p, pl.ord, hl->stride_layer, hl->stride_plane, hl->stride_block);
-    p.w0 = 0; p.w1 = pl.chunks;
-    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, full_grid(), stream));
-    return release_slot(ctx, slot, stream);
+  int variant = TALARIA_VARIANT_ZEROCOPY;     // gather / scatter: the copy kernel on a full grid
+  if (!img_on_device) {
+    variant = choose_variant(ctx, pl, hl, bt, n, to_image);
+    ctx->counters.last_variant = variant;
   }
-
-  // ---- choose how to cross the host link --------------------------------
-  BounceLane &ln = ctx->lane[to_image ? 0 : 1];
-  const int64_t dma_min = ctx->cfg.dma_min_bytes > 0 ? ctx->cfg.dma_min_bytes : (8ll << 20);
-  const int64_t seg_bytes = pl.run_chunks * pl.C;
-  const bool bounce_ok = (int64_t)ln.half >= pl.C;
-  int variant = ctx->cfg.variant;
-  if (variant == TALARIA_VARIANT_AUTO) {
-    variant = TALARIA_VARIANT_ZEROCOPY;
-    if (bounce_ok && payload >= dma_min && seg_bytes >= (256 << 10)) variant = TALARIA_VARIANT_BOUNCE;
-    // a table of few long runs of adjacent ids needs no kernel at all
-    if (payload >= dma_min && (hl->stride_block == pl.C || n == 1)) {
-      const int64_t copies = pl.L * pl.P * count_id_runs(bt, n);
-      if (copies <= 1024 && payload / copies >= (1 << 20)) variant = TALARIA_VARIANT_RUNS;
-    }
-  }
-  if (variant == TALARIA_VARIANT_BOUNCE && !bounce_ok) variant = TALARIA_VARIANT_ZEROCOPY;
-  ctx->counters.last_variant = variant;
 
   if (variant == TALARIA_VARIANT_ZEROCOPY) {
     p.img = (char *)img_dev;
     set_image_strides(p, pl.ord, hl->stride_layer, hl->stride_plane, hl->stride_block);
     p.w0 = 0; p.w1 = pl.chunks;
-    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, zc_grid(ctx), stream));
+    const int64_t grid_cap = img_on_device ? full_grid() : zc_grid(ctx);
+    if (fits_inline(pl.L * pl.P, n, pl.vec, p.img))
+      return launch_inline(ctx, to_image, p, pl.vec, grid_cap, kv->plane_base, pl.L * pl.P, bt, nullptr, n, stream);
+  }
+
+  // descriptor: plane pointers, then the table slice
+  const size_t ptr_bytes = (size_t)(pl.L * pl.P) * sizeof(void *);
+  const size_t desc_bytes = ptr_bytes + (size_t)n * sizeof(int32_t);
+  DescSlot *slot = nullptr;
+  if (variant != TALARIA_VARIANT_RUNS) {
+    TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+    memcpy(slot->h, kv->plane_base, ptr_bytes);
+    memcpy(slot->h + ptr_bytes, bt, (size_t)n * sizeof(int32_t));
+    TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+    p.plane_base = (const void *const *)slot->d;
+    p.table = (const int32_t *)(slot->d + ptr_bytes);
+  }
+
+  if (variant == TALARIA_VARIANT_ZEROCOPY) {
+    TAL_TRY(launch_dir(ctx, to_image, p, pl.vec, img_on_device ? full_grid() : zc_grid(ctx), stream));
     return release_slot(ctx, slot, stream);
   }
+  BounceLane &ln = ctx->lane[to_image ? 0 : 1];
 
   if (variant == TALARIA_VARIANT_RUNS) {
     // one copy-engine copy per (layer, plane, run of adjacent ids); needs no descriptor
@@ -379,7 +451,7 @@ static talaria_status_t kv_transfer(talaria_ctx *ctx, const talaria_kv_layout_t 
           i = j;
         }
       }
-    return release_slot(ctx, slot, stream);
+    return TALARIA_OK;
   }
 
   // ---- bounce: kernel <-> device bounce half <-> large copy-engine copies ----
@@ -468,20 +540,12 @@ static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_lay
   const size_t ptr_bytes = (size_t)(L * P) * sizeof(void *);
   const size_t off_bytes = (size_t)n * sizeof(int64_t);
   const size_t desc_bytes = ptr_bytes + off_bytes + (size_t)n * sizeof(int32_t);
-  DescSlot *slot;
-  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
-  memcpy(slot->h, kv->plane_base, ptr_bytes);
-  memcpy(slot->h + ptr_bytes, page_off, off_bytes);
-  memcpy(slot->h + ptr_bytes + off_bytes, bt, (size_t)n * sizeof(int32_t));
-  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
   const int64_t payload = n * slab;
   ctx->counters.payload_bytes += payload;
 
   KvCopyParams p{};
   p.num_blocks = kv->num_blocks;
   p.status = ctx->status_dev;
-  p.plane_base = (const void *const *)slot->d;
-  p.table = (const int32_t *)(slot->d + ptr_bytes + off_bytes);
   p.chunk_bytes = C;
   // digits: plane, layer, block -- the order of bytes inside consecutive slabs
   p.ord.e0 = P; p.ord.e1 = L;
@@ -505,6 +569,21 @@ static talaria_status_t kv_transfer_pages(talaria_ctx *ctx, const talaria_kv_lay
   }
   if (variant == TALARIA_VARIANT_BOUNCE && !bounce_ok) variant = TALARIA_VARIANT_ZEROCOPY;
   ctx->counters.last_variant = variant;
+
+  if (variant == TALARIA_VARIANT_ZEROCOPY && fits_inline(L * P, n, vec, pool_dev)) {
+    p.img = (char *)pool_dev;
+    p.sd[2] = 0;                              // the block's place comes from its page offset
+    p.w0 = 0; p.w1 = n * L * P;
+    return launch_inline(ctx, to_image, p, vec, zc_grid(ctx), kv->plane_base, L * P, bt, page_off, n, stream);
+  }
+  DescSlot *slot;
+  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+  memcpy(slot->h, kv->plane_base, ptr_bytes);
+  memcpy(slot->h + ptr_bytes, page_off, off_bytes);
+  memcpy(slot->h + ptr_bytes + off_bytes, bt, (size_t)n * sizeof(int32_t));
+  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+  p.plane_base = (const void *const *)slot->d;
+  p.table = (const int32_t *)(slot->d + ptr_bytes + off_bytes);
 
   if (variant == TALARIA_VARIANT_ZEROCOPY) {
     p.img = (char *)pool_dev;
@@ -789,15 +868,112 @@ static talaria_status_t batch_dup_check(talaria_ctx *ctx, const talaria_kv_layou
   return TALARIA_OK;
 }
 
+// Several sessions in one call.  Sessions that would each run the zero-copy kernel (the small
+// ones) and share their layer and plane strides are fused into ONE launch: the kernel sees
+// one image whose logical blocks are all the sessions' blocks back to back, each block
+// carrying the byte offset of its place in its own session's image -- the page-slab form of
+// the copy kernel.  Everything else (copy-engine variants, odd shapes) is enqueued in turn.
+// All arguments are checked before the first launch.
+static talaria_status_t kv_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv, const talaria_kv_xfer_t *x,
+                                 int32_t n_x, cudaStream_t stream, bool to_image) {
+  if (n_x < 0 || (n_x > 0 && !x) || !kv) return TALARIA_ERR_INVALID_ARG;
+  struct Member { int32_t s; Plan pl; char *img_dev; };
+  std::vector<Member> fuse;
+  std::vector<int32_t> solo;
+  for (int32_t s = 0; s < n_x; ++s) {
+    const talaria_kv_xfer_t &t = x[s];
+    if (t.n_blocks < 0 || t.first_block < 0) return TALARIA_ERR_INVALID_ARG;
+    if (t.n_blocks == 0) continue;
+    if (!t.block_table || !t.host) return TALARIA_ERR_INVALID_ARG;
+    Plan pl;
+    TAL_TRY(make_plan(kv, t.n_blocks, t.host, &t.hl, &pl));
+    const int32_t *bt = t.block_table + t.first_block;
+    TAL_TRY(validate_table(ctx, kv, bt, t.n_blocks, /*reject_dups=*/!to_image));
+    TAL_TRY(check_planes(ctx, kv, pl));
+    void *img_dev = nullptr;
+    TAL_TRY(mapped_range(ctx, t.host, t.hl.capacity_bytes, &img_dev));
+    const bool vec_ok = pl.vec != 0 && (uintptr_t)img_dev % 16 == 0;
+    if (vec_ok && choose_variant(ctx, pl, &t.hl, bt, t.n_blocks, to_image) == TALARIA_VARIANT_ZEROCOPY)
+      fuse.push_back(Member{s, pl, (char *)img_dev});
+    else
+      solo.push_back(s);
+  }
+  // ---- fused groups: members with equal (stride_layer, stride_plane) ------------------
+  std::vector<char> done(fuse.size(), 0);
+  std::vector<int64_t> page_off;
+  std::vector<int32_t> table;
+  for (size_t a = 0; a < fuse.size(); ++a) {
+    if (done[a]) continue;
+    const talaria_host_layout_t &ha = x[fuse[a].s].hl;
+    const Plan &pa = fuse[a].pl;
+    // a dimension of extent 1 has no meaningful stride: compare only what addresses use
+    auto same = [&](const talaria_host_layout_t &h) {
+      return (pa.L == 1 || h.stride_layer == ha.stride_layer) && (pa.P == 1 || h.stride_plane == ha.stride_plane);
+    };
+    char *base = fuse[a].img_dev;
+    int vec = 32;
+    for (size_t b = a; b < fuse.size(); ++b)
+      if (!done[b] && same(x[fuse[b].s].hl)) base = std::min(base, fuse[b].img_dev);
+    page_off.clear();
+    table.clear();
+    int32_t members = 0;
+    for (size_t b = a; b < fuse.size(); ++b) {
+      if (done[b] || !same(x[fuse[b].s].hl)) continue;
+      done[b] = 1;
+      ++members;
+      const talaria_kv_xfer_t &t = x[fuse[b].s];
+      vec = std::min(vec, fuse[b].pl.vec);
+      if ((uintptr_t)fuse[b].img_dev % 32 != 0) vec = std::min(vec, 16);
+      for (int64_t i = 0; i < t.n_blocks; ++i) {
+        page_off.push_back((int64_t)(fuse[b].img_dev - base) + i * t.hl.stride_block);
+        table.push_back(t.block_table[t.first_block + i]);
+      }
+    }
+    const int64_t n = (int64_t)table.size(), L = pa.L, P = pa.P, C = pa.C;
+    KvCopyParams p{};
+    p.num_blocks = kv->num_blocks;
+    p.status = ctx->status_dev;
+    p.chunk_bytes = C;
+    p.img = base;
+    // digits: plane, layer, block -- the block's place comes from its offset
+    p.ord.e0 = P; p.ord.e1 = L;
+    p.ord.lp_coef[0] = 1; p.ord.lp_coef[1] = (int32_t)P; p.ord.lp_coef[2] = 0;
+    p.ord.i_coef[0] = 0; p.ord.i_coef[1] = 0; p.ord.i_coef[2] = 1;
+    p.sd[0] = P == 1 ? 0 : ha.stride_plane; p.sd[1] = L == 1 ? 0 : ha.stride_layer; p.sd[2] = 0;
+    p.w0 = 0; p.w1 = n * L * P;
+    ctx->counters.payload_bytes += n * L * P * C;
+    ctx->counters.last_variant = TALARIA_VARIANT_ZEROCOPY;
+    if (fits_inline(L * P, n, vec, base)) {
+      TAL_TRY(launch_inline(ctx, to_image, p, vec, zc_grid(ctx), kv->plane_base, L * P, table.data(), page_off.data(), n, stream));
+      continue;
+    }
+    const size_t ptr_bytes = (size_t)(L * P) * sizeof(void *), off_bytes = (size_t)n * sizeof(int64_t);
+    const size_t desc_bytes = ptr_bytes + off_bytes + (size_t)n * sizeof(int32_t);
+    DescSlot *slot;
+    TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+    memcpy(slot->h, kv->plane_base, ptr_bytes);
+    memcpy(slot->h + ptr_bytes, page_off.data(), off_bytes);
+    memcpy(slot->h + ptr_bytes + off_bytes, table.data(), (size_t)n * sizeof(int32_t));
+    TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+    p.plane_base = (const void *const *)slot->d;
+    p.page_off = (const int64_t *)(slot->d + ptr_bytes);
+    p.table = (const int32_t *)(slot->d + ptr_bytes + off_bytes);
+    TAL_TRY(launch_dir(ctx, to_image, p, vec, zc_grid(ctx), stream));
+    TAL_TRY(release_slot(ctx, slot, stream));
+    (void)members;
+  }
+  // ---- the rest, one after the other ------------------------------------------------------
+  for (int32_t s : solo)
+    TAL_TRY(kv_transfer(ctx, kv, x[s].block_table, x[s].first_block, x[s].n_blocks, x[s].host, &x[s].hl, stream,
+                        to_image, false));
+  return TALARIA_OK;
+}
+
 extern "C" talaria_status_t talaria_kv_offload_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
                                                      const talaria_kv_xfer_t *xfers, int32_t n_xfers,
                                                      void *stream) {
   TAL_ENTER(ctx);
-  if (n_xfers < 0 || (n_xfers > 0 && !xfers)) return TALARIA_ERR_INVALID_ARG;
-  for (int32_t s = 0; s < n_xfers; ++s)
-    TAL_TRY(kv_transfer(ctx, kv, xfers[s].block_table, xfers[s].first_block, xfers[s].n_blocks,
-                        xfers[s].host, &xfers[s].hl, (cudaStream_t)stream, true, false));
-  return TALARIA_OK;
+  return kv_batch(ctx, kv, xfers, n_xfers, (cudaStream_t)stream, true);
 }
 
 extern "C" talaria_status_t talaria_kv_restore_batch(talaria_ctx *ctx, const talaria_kv_layout_t *kv,
@@ -806,8 +982,5 @@ extern "C" talaria_status_t talaria_kv_restore_batch(talaria_ctx *ctx, const tal
   TAL_ENTER(ctx);
   if (n_xfers < 0 || (n_xfers > 0 && !xfers)) return TALARIA_ERR_INVALID_ARG;
   TAL_TRY(batch_dup_check(ctx, kv, xfers, n_xfers));
-  for (int32_t s = 0; s < n_xfers; ++s)
-    TAL_TRY(kv_transfer(ctx, kv, xfers[s].block_table, xfers[s].first_block, xfers[s].n_blocks,
-                        xfers[s].host, &xfers[s].hl, (cudaStream_t)stream, false, false));
-  return TALARIA_OK;
+  return kv_batch(ctx, kv, xfers, n_xfers, (cudaStream_t)stream, false);
 }

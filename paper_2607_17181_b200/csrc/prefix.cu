@@ -537,41 +537,64 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
   if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
   if (n_pairs == 0) return TALARIA_OK;
   if (!cont_offsets || !sess_offsets || !h_results) return TALARIA_ERR_INVALID_ARG;
-  const int64_t c0 = cont_offsets[0], s0 = sess_offsets[0];
-  const int64_t nc = cont_offsets[n_pairs] - c0, ns = sess_offsets[n_pairs] - s0;
-  if (nc < 0 || ns < 0 || (nc > 0 && !h_cont) || (ns > 0 && !h_sess)) return TALARIA_ERR_INVALID_ARG;
-  int64_t cb = 0, sb = 0;
-  std::vector<int64_t> co(n_pairs + 1), so(n_pairs + 1);
-  for (int32_t q = 0; q <= n_pairs; ++q) {
-    co[q] = cont_offsets[q] - c0;
-    so[q] = sess_offsets[q] - s0;
-    if (q < n_pairs) {
-      int64_t Tc = cont_offsets[q + 1] - cont_offsets[q], Ts = sess_offsets[q + 1] - sess_offsets[q];
-      if (Tc < 0 || Ts < 0) return TALARIA_ERR_INVALID_ARG;
-      cb += Tc / B;
-      sb += Ts / B;
-    }
-  }
+  for (int32_t q = 0; q < n_pairs; ++q)
+    if (cont_offsets[q + 1] < cont_offsets[q] || sess_offsets[q + 1] < sess_offsets[q] || cont_offsets[q] < 0 ||
+        sess_offsets[q] < 0)
+      return TALARIA_ERR_INVALID_ARG;
+  if ((cont_offsets[n_pairs] > cont_offsets[0] && !h_cont) || (sess_offsets[n_pairs] > sess_offsets[0] && !h_sess))
+    return TALARIA_ERR_INVALID_ARG;
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
-  const size_t o_cont = 0, o_sess = o_cont + up((size_t)nc * 4), o_sh = o_sess + up((size_t)ns * 4),
-               o_ch = o_sh + up(h_sess_hashes ? (size_t)sb * 8 : 0), o_res = o_ch + up((size_t)cb * 8),
-               total = o_res + up((size_t)n_pairs * sizeof(talaria_match_t));
-  TAL_TRY(grow(ctx, &ctx->host_tok, total));
-  char *d = ctx->host_tok.p;
-  if (nc) TAL_CUDA(ctx, cudaMemcpyAsync(d + o_cont, h_cont + c0, (size_t)nc * 4, cudaMemcpyHostToDevice, stream));
-  if (ns) TAL_CUDA(ctx, cudaMemcpyAsync(d + o_sess, h_sess + s0, (size_t)ns * 4, cudaMemcpyHostToDevice, stream));
-  if (h_sess_hashes && sb)
-    TAL_CUDA(ctx, cudaMemcpyAsync(d + o_sh, h_sess_hashes, (size_t)sb * 8, cudaMemcpyHostToDevice, stream));
-  ctx->counters.memcpy_calls += 3;
-  TAL_TRY(prefix_launch(ctx, n_pairs, (const int32_t *)(d + o_cont), co.data(), (const int32_t *)(d + o_sess),
-                        so.data(), h_sess_hashes ? (const uint64_t *)(d + o_sh) : nullptr, B, seed,
-                        (uint64_t *)(d + o_ch), (talaria_match_t *)(d + o_res), stream));
-  if (h_cont_hashes_out && cb)
-    TAL_CUDA(ctx, cudaMemcpyAsync(h_cont_hashes_out, d + o_ch, (size_t)cb * 8, cudaMemcpyDeviceToHost, stream));
-  TAL_CUDA(ctx, cudaMemcpyAsync(h_results, d + o_res, (size_t)n_pairs * sizeof(talaria_match_t),
-                                cudaMemcpyDeviceToHost, stream));
-  ctx->counters.memcpy_calls += 2;
-  TAL_CUDA(ctx, cudaStreamSynchronize(stream));
+  const size_t cap = ctx->host_tok.cap;
+  char *const dev = ctx->host_tok.p, *const pin = ctx->match_pin;
+  std::vector<int64_t> co, so;
+  int64_t sb_before = 0, cb_before = 0;           // blocks of the pairs already done (positions in the users' hash arrays)
+  for (int32_t q0 = 0; q0 < n_pairs;) {
+    // the longest run of whole pairs whose inputs and outputs fit the staging
+    int32_t q1 = q0;
+    int64_t nc = 0, ns = 0, cb = 0, sb = 0;
+    while (q1 < n_pairs) {
+      const int64_t Tc = cont_offsets[q1 + 1] - cont_offsets[q1], Ts = sess_offsets[q1 + 1] - sess_offsets[q1];
+      const size_t need = up((size_t)(nc + Tc) * 4) + up((size_t)(ns + Ts) * 4) +
+                          up(h_sess_hashes ? (size_t)(sb + Ts / B) * 8 : 0) + up((size_t)(cb + Tc / B) * 8) +
+                          up((size_t)(q1 + 1 - q0) * sizeof(talaria_match_t));
+      if (need > cap) break;
+      nc += Tc; ns += Ts; cb += Tc / B; sb += Ts / B;
+      ++q1;
+    }
+    if (q1 == q0) return TALARIA_ERR_EXTENT;       // one pair alone is larger than the staging
+    const int32_t m = q1 - q0;
+    const size_t o_cont = 0, o_sess = o_cont + up((size_t)nc * 4), o_sh = o_sess + up((size_t)ns * 4),
+                 o_ch = o_sh + up(h_sess_hashes ? (size_t)sb * 8 : 0), o_res = o_ch + up((size_t)cb * 8),
+                 o_end = o_res + up((size_t)m * sizeof(talaria_match_t));
+    const int64_t c0 = cont_offsets[q0], s0 = sess_offsets[q0];
+    co.resize((size_t)m + 1);
+    so.resize((size_t)m + 1);
+    for (int32_t q = 0; q <= m; ++q) {
+      co[(size_t)q] = cont_offsets[q0 + q] - c0;
+      so[(size_t)q] = sess_offsets[q0 + q] - s0;
+    }
+    // gather the inputs into the pinned staging; one copy takes them to the device
+    if (nc) memcpy(pin + o_cont, h_cont + c0, (size_t)nc * 4);
+    if (ns) memcpy(pin + o_sess, h_sess + s0, (size_t)ns * 4);
+    if (h_sess_hashes && sb) memcpy(pin + o_sh, h_sess_hashes + sb_before, (size_t)sb * 8);
+    if (o_ch) {
+      TAL_CUDA(ctx, cudaMemcpyAsync(dev, pin, o_ch, cudaMemcpyHostToDevice, stream));
+      ctx->counters.memcpy_calls++;
+    }
+    TAL_TRY(prefix_launch(ctx, m, (const int32_t *)(dev + o_cont), co.data(), (const int32_t *)(dev + o_sess),
+                          so.data(), h_sess_hashes ? (const uint64_t *)(dev + o_sh) : nullptr, B, seed,
+                          (uint64_t *)(dev + o_ch), (talaria_match_t *)(dev + o_res), stream));
+    // hashes and results come back in one copy
+    const size_t out_from = (h_cont_hashes_out && cb) ? o_ch : o_res;
+    TAL_CUDA(ctx, cudaMemcpyAsync(pin + out_from, dev + out_from, o_end - out_from, cudaMemcpyDeviceToHost, stream));
+    ctx->counters.memcpy_calls++;
+    TAL_CUDA(ctx, cudaStreamSynchronize(stream));
+    if (h_cont_hashes_out && cb) memcpy(h_cont_hashes_out + cb_before, pin + o_ch, (size_t)cb * 8);
+    memcpy(h_results + q0, pin + o_res, (size_t)m * sizeof(talaria_match_t));
+    sb_before += sb;
+    cb_before += cb;
+    q0 = q1;
+  }
   return TALARIA_OK;
 }
 

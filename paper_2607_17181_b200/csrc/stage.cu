@@ -167,6 +167,17 @@ static talaria_status_t classify_plan(const talaria_copy_t *plan, int64_t n, con
   return TALARIA_OK;
 }
 
+// One merged host-sourced run, as copy-engine copies of bounded size on the reload stream: a
+// restore running on the context's other streams gets the link between two pieces.
+static talaria_status_t enqueue_reload(talaria_ctx *ctx, const char *h, char *d, int64_t bytes) {
+  for (int64_t at = 0; at < bytes; at += kReloadPiece) {
+    const size_t n = (size_t)std::min(kReloadPiece, bytes - at);
+    TAL_CUDA(ctx, cudaMemcpyAsync(d + at, h + at, n, cudaMemcpyHostToDevice, ctx->reload_stream));
+    ctx->counters.memcpy_calls++;
+  }
+  return TALARIA_OK;
+}
+
 // Every destination, and every staged source that will be read, must lie inside one device
 // allocation for its whole length.  from_host (nullable): entries whose staged source is not read.
 static talaria_status_t check_device_ranges(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
@@ -213,11 +224,10 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   TAL_TRY(check_device_ranges(ctx, plan, n, from_host.data()));
   // The internal stream forks from the caller's stream BEFORE the D2D kernel is launched, so
   // the host-sourced copies depend only on earlier work and run next to the kernel.
-  BounceLane &ln = ctx->lane[1];
   const bool forked = !runs.empty();
   if (forked) {
-    TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
-    TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
+    TAL_CUDA(ctx, cudaEventRecord(ctx->reload_fork, stream));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(ctx->reload_stream, ctx->reload_fork, 0));
   }
   // ---- D2D leg ---------------------------------------------------------------
   if (n_clean > 0 && st.d2d_bytes > 0) {
@@ -253,12 +263,9 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   }
   // ---- H2D leg, part 2: enqueued second, so the kernel is already running meanwhile
   if (forked) {
-    for (const HostRun &r : runs) {
-      TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
-      ctx->counters.memcpy_calls++;
-    }
-    TAL_CUDA(ctx, cudaEventRecord(ln.done[0], ln.s[0]));
-    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[0], 0));
+    for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    TAL_CUDA(ctx, cudaEventRecord(ctx->reload_done, ctx->reload_stream));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->reload_done, 0));
   }
   ctx->counters.payload_bytes += st.d2d_bytes + st.h2d_bytes;
   if (stats) *stats = st;
@@ -392,10 +399,9 @@ static talaria_status_t plan_run(talaria_ctx *ctx, talaria_stage_plan *sp, const
     ctx->counters.memcpy_calls++;
     d_bitmap = sp->d_dirty;
   }
-  BounceLane &ln = ctx->lane[1];
   if (!runs.empty()) {
-    TAL_CUDA(ctx, cudaEventRecord(ln.fork, stream));
-    TAL_CUDA(ctx, cudaStreamWaitEvent(ln.s[0], ln.fork, 0));
+    TAL_CUDA(ctx, cudaEventRecord(ctx->reload_fork, stream));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(ctx->reload_stream, ctx->reload_fork, 0));
   }
   if (sp->tiles > 0 && st.d2d_bytes > 0) {
     StageParams p{(const StageEntry *)sp->d_desc, (const int32_t *)(sp->d_desc + sp->ent_bytes), n, sp->tiles, d_bitmap};
@@ -406,12 +412,9 @@ static talaria_status_t plan_run(talaria_ctx *ctx, talaria_stage_plan *sp, const
   // (the device bitmap is rewritten by the next run's upload, which the caller orders after
   // this kernel: runs of one prepared plan share a stream or are chained with events)
   if (!runs.empty()) {
-    for (const HostRun &r : runs) {
-      TAL_CUDA(ctx, cudaMemcpyAsync(r.d, r.h, (size_t)r.bytes, cudaMemcpyHostToDevice, ln.s[0]));
-      ctx->counters.memcpy_calls++;
-    }
-    TAL_CUDA(ctx, cudaEventRecord(ln.done[0], ln.s[0]));
-    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ln.done[0], 0));
+    for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    TAL_CUDA(ctx, cudaEventRecord(ctx->reload_done, ctx->reload_stream));
+    TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->reload_done, 0));
   }
   ctx->counters.payload_bytes += st.d2d_bytes + st.h2d_bytes;
   if (stats) *stats = st;

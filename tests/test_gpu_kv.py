@@ -166,6 +166,64 @@ def test_registered_host_memory_and_batch_forms(ctxs):
         ctx.host_unregister(raw)
 
 
+@pytest.mark.parametrize("order", ["PF", "LF"])
+def test_batch_of_many_small_sessions_is_one_fused_launch(ctxs, order):
+    ctx = ctxs[tb.VARIANT_AUTO]
+    shape, nb = wl.TINY, 1536
+    g = wl.rng(18)
+    planes = wl.kv_pool(g, shape, nb)
+    pool = DevicePool(shape, planes)
+    expect = [p.copy() for p in planes]
+    for sizes in ([1] * 64, [3] * 40 + [1] * 50, [5, 1, 9, 2, 30, 1, 1, 7] * 10):     # <= 256 blocks inline, then beyond
+        tables = wl.disjoint_tables(g, nb, sizes)
+        new_tables = wl.disjoint_tables(g, nb, sizes, exclude=np.concatenate(tables))[::-1]
+        imgs = [GuardedPinned(n * shape.bytes_per_block) for n in sizes]
+        xf = [(bt, 0, bt.size, im.ptr, tb.host_layout(wl.dense_strides(shape, bt.size, order), im.n))
+              for bt, im in zip(tables, imgs)]
+        ctx.reset_counters()
+        ctx.kv_offload_batch(pool.kv, xf)
+        ctx.sync()
+        c = ctx.get_counters()
+        # page-first images all share their layer / plane strides; layer-first ones only at equal block counts
+        per_group = [sum(sizes)] if order == "PF" else [sum(n for n in sizes if n == k) for k in set(sizes)]
+        groups = len(per_group)
+        assert c.kernel_launches == groups, (order, sizes[:4], c.kernel_launches)
+        assert c.memcpy_calls == sum(1 for b in per_group if b > 256)               # up to 256 blocks: no upload
+        for bt, im in zip(tables, imgs):
+            want = np.zeros(im.n, np.uint8)
+            orc.kv_offload(oshape(shape), expect, bt, 0, bt.size, want, wl.dense_strides(shape, bt.size, order))
+            assert np.array_equal(im.np, want) and im.guards_ok()
+        ctx.reset_counters()
+        ctx.kv_restore_batch(pool.kv, [(bt2, 0, bt2.size, im.ptr, x[4]) for bt2, im, x in zip(new_tables[::-1], imgs, xf)])
+        ctx.sync()
+        assert ctx.get_counters().kernel_launches == groups
+        for bt2, im in zip(new_tables[::-1], imgs):
+            orc.kv_restore(oshape(shape), expect, bt2, 0, bt2.size, im.np, wl.dense_strides(shape, bt2.size, order))
+        for a, b in zip(pool.read(), expect):
+            assert np.array_equal(a, b)
+        assert pool.guards_ok()
+
+
+def test_small_transfers_carry_their_descriptor_in_the_launch(ctxs):
+    ctx = ctxs[tb.VARIANT_ZEROCOPY]
+    shape, nb = wl.TINY, 64
+    g = wl.rng(19)
+    planes = wl.kv_pool(g, shape, nb)
+    pool = DevicePool(shape, planes)
+    for n, uploads in ((1, 0), (256 if nb >= 256 else nb, 0)):
+        bt = wl.disjoint_tables(g, nb, [n])[0]
+        img = GuardedPinned(n * shape.bytes_per_block)
+        strides = wl.dense_strides(shape, n, "PF")
+        ctx.reset_counters()
+        ctx.kv_offload(pool.kv, bt, 0, n, img.ptr, tb.host_layout(strides, img.n))
+        ctx.sync()
+        c = ctx.get_counters()
+        assert (c.kernel_launches, c.memcpy_calls) == (1, uploads)
+        want = np.zeros(img.n, np.uint8)
+        orc.kv_offload(oshape(shape), planes, bt, 0, n, want, strides)
+        assert np.array_equal(img.np, want) and img.guards_ok()
+
+
 def test_argument_errors_never_reach_the_gpu(ctxs):
     ctx = ctxs[tb.VARIANT_AUTO]
     shape, nb = wl.TINY, 32

@@ -164,6 +164,44 @@ def test_host_entry_point_matches_oracle(ctx):
             at += hc.size
 
 
+def test_host_entry_point_splits_batches_larger_than_its_staging():
+    # 1 MiB of staging (the minimum): the batch below needs several sub-batches of whole pairs
+    small = tb.Talaria(0, host_match_bytes=1 << 20)
+    try:
+        g = wl.rng(510)
+        pairs = []
+        for _ in range(40):
+            ts, tc = int(g.integers(0, 20_000)), int(g.integers(0, 20_000))
+            s = wl.tokens(g, ts)
+            pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1))), s))
+        cont = np.concatenate([c for c, _ in pairs]); sess = np.concatenate([s for _, s in pairs])
+        co = np.cumsum([0] + [c.size for c, _ in pairs]); so = np.cumsum([0] + [s.size for _, s in pairs])
+        assert (cont.size + sess.size) * 4 > 3 * (1 << 20)
+        for stored in (False, True):
+            hs = np.concatenate([orc.block_hash(s, 16, SEED) for _, s in pairs]) if stored else None
+            out_h = np.zeros(sum(c.size // 16 for c, _ in pairs), np.uint64)
+            res = np.zeros(len(pairs), tb.MATCH_DTYPE)
+            before = small.get_counters().kernel_launches
+            small.prefix_match_host(len(pairs), cont, co, sess, so, hs, 16, SEED, out_h, res)
+            assert small.get_counters().kernel_launches - before >= 3          # really several sub-batches
+            at = 0
+            for q, (c, s) in enumerate(pairs):
+                m, hc = orc.prefix_match(c, s, 16, SEED)
+                assert (int(res[q]["lcp_tokens"]), int(res[q]["matched_blocks"]), int(res[q]["reusable_tokens"]),
+                        int(res[q]["hash_token_disagree"])) == (m.lcp_tokens, m.matched_blocks, m.reusable_tokens, 0)
+                assert np.array_equal(out_h[at:at + hc.size], hc)
+                at += hc.size
+        # a single pair that cannot fit is refused; nothing is allocated to make room
+        big = wl.tokens(g, 200_000)
+        free_before = torch.cuda.mem_get_info()[0]
+        with pytest.raises(tb.TalariaError) as e:
+            small.prefix_match_host(1, big, [0, big.size], big, [0, big.size], None, 16, SEED, None, np.zeros(1, tb.MATCH_DTYPE))
+        assert e.value.status == tb.ERR_EXTENT
+        assert torch.cuda.mem_get_info()[0] == free_before
+    finally:
+        small.destroy()
+
+
 def test_prefix_agree_host_arithmetic():
     g = wl.rng(506)
     for _ in range(100):
