@@ -1,4 +1,4 @@
-"""Session-replay driver: the eviction policy around the library calls.
+"""Session-replay driver: the residency policy around the library calls.
 
 The library moves bytes; which session is evicted, when a prefix is restored and
 where new blocks come from is the caller's policy (the paper's instance-local
@@ -7,15 +7,26 @@ sessions against one paged KV pool of fixed capacity:
 
   * every group of calls is prefix-matched in one batched call against the
     sessions' stored streams (App. A) -- `talaria_prefix_match_host`;
+  * when a call finishes, its newly aligned (full) blocks are checkpointed to pinned
+    host memory on a checkpoint stream, asynchronously, one extent per call
+    (Sec. 4.1 / 4.3: checkpoint when a request finishes) -- `talaria_kv_offload`
+    with a `first_block / n_blocks` sub-range;
   * a returning session whose KV is still in the pool keeps the matched blocks and
-    frees the rest; one whose KV was moved to the host gets new blocks and the
-    matched prefix is restored into them (Sec. 4.3) -- `talaria_kv_restore_batch`;
+    frees the rest (checkpoint extents beyond the match are cut back); one whose KV
+    lives only on the host gets new blocks and the matched prefix is restored into
+    them, extent by extent (Sec. 4.3) -- `talaria_kv_restore_batch`; the restored
+    blocks need no new checkpoint;
   * when the pool cannot hold a call, whole sessions are evicted in LRU order
-    (ties: lower session id) to pinned host images -- `talaria_kv_offload_batch`;
-    when the host budget is exhausted the oldest host images are dropped and the
-    next call of that session recomputes everything ("host-cache capacity miss");
+    (ties: lower session id).  Eviction drains the victim's checkpoint event and
+    copies only what is not on the host yet -- normally the partial tail block
+    (App. B: the barrier usually waits only for the final tail blocks);
+    when the host budget is exhausted the oldest host-only sessions are dropped and
+    their next call recomputes everything ("host-cache capacity miss");
   * the KV of the unmatched tail is "computed": synthetic bytes are scattered
     into the new blocks -- `talaria_kv_scatter`.
+
+`checkpoint="eviction"` is the simpler policy with no background checkpoints: the
+whole session is copied when it is evicted.
 
 Every byte-moving step is appended to `log` so a test can replay the same steps on
 the CPU oracle; this module itself never imports the oracle.
@@ -34,15 +45,29 @@ from . import workloads as wl
 
 
 @dataclass
+class Extent:
+    """Blocks [first, first + n) of a session, checkpointed in one call, as a dense host image."""
+    first: int
+    n: int
+    image: object                 # pinned host tensor of n * bytes_per_block
+    hl: object                    # its layout
+    cap: int                      # blocks the image was sized for (n may be cut back later)
+
+
+@dataclass
 class SessionState:
     sid: int
     tokens: np.ndarray = field(default_factory=lambda: np.zeros(0, np.int32))
     hashes: np.ndarray = field(default_factory=lambda: np.zeros(0, np.uint64))
     table: Optional[np.ndarray] = None        # block ids while resident in the pool
     where: str = "none"                       # "device" | "host" | "none"
-    image: object = None                      # pinned host tensor while where == "host"
-    image_blocks: int = 0
+    extents: List[Extent] = field(default_factory=list)
+    event: object = None                      # end of the last checkpoint copy (torch.cuda.Event) or None
     last_use: int = -1
+
+    @property
+    def host_blocks(self) -> int:
+        return self.extents[-1].first + self.extents[-1].n if self.extents else 0
 
 
 @dataclass
@@ -53,11 +78,17 @@ class ReplayStats:
     recomputes: int = 0
     capacity_misses: int = 0
     evictions: int = 0
-    offload_bytes: int = 0
+    offload_bytes: int = 0        # all device-to-host KV bytes (checkpoints and evictions)
     restore_bytes: int = 0
+    checkpoint_bytes: int = 0     # of which background checkpoints
+    checkpoints_skipped: int = 0  # no host budget at checkpoint time
+    evict_bytes_already_on_host: int = 0
+    evict_bytes_copied: int = 0
+    evict_stall_s: float = 0.0    # host time an eviction blocked: drain of the checkpoint event + tail copy
+    evict_stalls: List[float] = field(default_factory=list)
     reused_tokens: int = 0
     prompt_tokens: int = 0
-    offload_s: float = 0.0        # host wall time of the batched calls, drained
+    offload_s: float = 0.0        # host wall time of the synchronous transfer calls, drained
     restore_s: float = 0.0
     match_s: float = 0.0
     match_calls: int = 0
@@ -68,13 +99,16 @@ class ReplayDriver:
     def __init__(self, ctx: tb.Talaria, shape: wl.KvShape, kv, pool_blocks: int, host_budget_bytes: int,
                  seed: int, content: Callable[[int, int, int], np.ndarray], alloc_pinned: Callable[[int], object],
                  to_device: Callable[[np.ndarray], object], order: str = "PF", log: Optional[list] = None,
-                 free_pinned: Optional[Callable[[object], None]] = None):
+                 free_pinned: Optional[Callable[[object], None]] = None, checkpoint: str = "incremental"):
         """content(session, call_index, nbytes) -> uint8 array: the synthetic KV of a call's new blocks.
         alloc_pinned(nbytes) -> pinned host tensor; free_pinned(tensor) gives it back (optional);
-        to_device(array) -> device tensor (memory plumbing)."""
+        to_device(array) -> device tensor (memory plumbing).
+        checkpoint: "incremental" (after every call, asynchronously) or "eviction" (whole session when evicted)."""
+        import torch
+        assert checkpoint in ("incremental", "eviction")
         self.ctx, self.shape, self.kv = ctx, shape, kv
         self.pool_blocks, self.host_budget = pool_blocks, host_budget_bytes
-        self.seed, self.order = seed, order
+        self.seed, self.order, self.checkpoint = seed, order, checkpoint
         self.content, self.alloc_pinned, self.to_device = content, alloc_pinned, to_device
         self.free_pinned = free_pinned
         self.free: List[int] = list(range(pool_blocks))      # min-heap: low addresses are reused first
@@ -84,6 +118,8 @@ class ReplayDriver:
         self.clock = 0
         self.stats = ReplayStats()
         self.log = log if log is not None else []
+        self._torch = torch
+        self.ckpt_stream = torch.cuda.Stream()
 
     # ------------------------------------------------------------ allocation
     def _alloc(self, n: int) -> np.ndarray:
@@ -93,59 +129,132 @@ class ReplayDriver:
         for b in ids:
             heapq.heappush(self.free, int(b))
 
-    def _drop_host(self, s: SessionState):
-        self.host_bytes -= s.image_blocks * self.shape.bytes_per_block
-        if self.free_pinned is not None and s.image is not None:
-            self.free_pinned(s.image)
-        s.image, s.image_blocks, s.where = None, 0, "none"
+    # ------------------------------------------------------------- host side
+    def _extent_bytes(self, e: Extent) -> int:
+        return e.cap * self.shape.bytes_per_block
 
+    def _free_extent(self, e: Extent):
+        self.host_bytes -= self._extent_bytes(e)
+        if self.free_pinned is not None:
+            self.free_pinned(e.image)
+
+    def _drop_host(self, s: SessionState):
+        """Forget everything the host holds of this session."""
+        if s.event is not None:
+            s.event.synchronize()                 # a copy into these images may still be running
+            s.event = None
+        for e in s.extents:
+            self._free_extent(e)
+        s.extents = []
+        if s.where == "host":
+            s.where = "none"
+
+    def _truncate_host(self, s: SessionState, keep: int):
+        """Keep only the checkpoints of blocks [0, keep): the rest describes KV that is being replaced."""
+        if s.host_blocks <= keep:
+            return
+        if s.event is not None:
+            s.event.synchronize()
+            s.event = None
+        kept = []
+        for e in s.extents:
+            if e.first >= keep:
+                self._free_extent(e)
+            else:
+                e.n = min(e.n, keep - e.first)
+                kept.append(e)
+        s.extents = kept
+        self.log.append(("truncate", s.sid, keep))
+
+    def _host_room(self, nbytes: int, busy: set) -> bool:
+        """Make room in the host budget by dropping the oldest host-only sessions."""
+        while self.host_bytes + nbytes > self.host_budget:
+            old = sorted((h for h in self.sessions.values() if h.where == "host" and h.sid not in busy),
+                         key=lambda h: (h.last_use, h.sid))
+            if not old:
+                return False
+            self._drop_host(old[0])
+            self.log.append(("drop_host", old[0].sid))
+        return True
+
+    def _new_extent(self, s: SessionState, first: int, n: int) -> Extent:
+        nbytes = n * self.shape.bytes_per_block
+        image = self.alloc_pinned(nbytes)
+        hl = tb.host_layout(wl.dense_strides(self.shape, n, self.order), nbytes)
+        e = Extent(first, n, image, hl, n)
+        self.host_bytes += nbytes
+        s.extents.append(e)
+        return e
+
+    def _checkpoint(self, s: SessionState, busy: set, fill_done):
+        """Asynchronously checkpoint the session's newly aligned (full) blocks."""
+        full = s.tokens.size // self.shape.block_tokens
+        first = s.host_blocks
+        n = full - first
+        if n <= 0:
+            return
+        if not self._host_room(n * self.shape.bytes_per_block, busy | {s.sid}):
+            self.stats.checkpoints_skipped += 1
+            return
+        e = self._new_extent(s, first, n)
+        self.ckpt_stream.wait_event(fill_done)
+        self.ctx.kv_offload(self.kv, s.table, first, n, e.image, e.hl, stream=self.ckpt_stream)
+        s.event = self._torch.cuda.Event()
+        s.event.record(self.ckpt_stream)
+        self.stats.checkpoint_bytes += n * self.shape.bytes_per_block
+        self.stats.offload_bytes += n * self.shape.bytes_per_block
+        self.log.append(("checkpoint", s.sid, first, s.table[first:first + n].copy()))
+
+    # --------------------------------------------------------------- eviction
     def _make_room(self, need: int, busy: set):
         """Evict whole sessions, least recently used first, until `need` blocks are free."""
         if len(self.free) >= need:
             return
         victims = sorted((s for s in self.sessions.values() if s.where == "device" and s.sid not in busy),
                          key=lambda s: (s.last_use, s.sid))
-        xfers, chosen, freed = [], [], len(self.free)
+        freed = len(self.free)
         for s in victims:
             if freed >= need:
                 break
-            n = len(s.table)
-            nbytes = n * self.shape.bytes_per_block
-            # host budget: drop the oldest host images first; if it still does not fit, the KV is lost
-            while self.host_bytes + nbytes > self.host_budget:
-                old = sorted((h for h in self.sessions.values() if h.where == "host" and h.sid not in busy),
-                             key=lambda h: (h.last_use, h.sid))
-                if not old:
-                    break
-                self._drop_host(old[0])
-                self.log.append(("drop_host", old[0].sid))
-            if self.host_bytes + nbytes <= self.host_budget:
-                s.image = self.alloc_pinned(nbytes)
-                s.image_blocks = n
-                hl = tb.host_layout(wl.dense_strides(self.shape, n, self.order), nbytes)
-                xfers.append((s.table.copy(), 0, n, s.image, hl))
-                self.host_bytes += nbytes
-            chosen.append(s)
-            freed += n
-        if freed < need:
-            raise RuntimeError("pool too small for this call even after evicting every other session")
-        if xfers:
             t0 = time.perf_counter()
-            self.ctx.kv_offload_batch(self.kv, xfers)
-            self.ctx.sync()                                   # drain before the blocks are reused (App. B)
-            self.stats.offload_s += time.perf_counter() - t0
-            self.stats.offload_bytes += sum(x[2] for x in xfers) * self.shape.bytes_per_block
-        for s in chosen:
-            kept = s.image is not None
-            self.log.append(("offload" if kept else "evict_lost", s.sid, s.table.copy()))
+            n_all = len(s.table)
+            first = s.host_blocks
+            rest = n_all - first                                  # not on the host yet (normally the tail block)
+            kept = True
+            if rest > 0:
+                if self._host_room(rest * self.shape.bytes_per_block, busy | {s.sid}):
+                    e = self._new_extent(s, first, rest)
+                    self.ctx.kv_offload(self.kv, s.table, first, rest, e.image, e.hl)
+                    self.stats.offload_bytes += rest * self.shape.bytes_per_block
+                    self.stats.evict_bytes_copied += rest * self.shape.bytes_per_block
+                    self.log.append(("checkpoint", s.sid, first, s.table[first:first + rest].copy()))
+                else:
+                    kept = False                                  # no host room: this session's KV is lost
+            # switch barrier for this session: its checkpoint copies and the tail copy are done
+            if s.event is not None:
+                s.event.synchronize()
+                s.event = None
+            self.ctx.sync()
+            dt = time.perf_counter() - t0
+            self.stats.evict_stall_s += dt
+            self.stats.evict_stalls.append(dt)
+            self.stats.offload_s += dt
+            self.stats.evict_bytes_already_on_host += first * self.shape.bytes_per_block
+            if not kept:
+                self._drop_host(s)
+            self.log.append(("evict" if kept else "evict_lost", s.sid, s.table.copy()))
             self._release(s.table)
             s.table = None
             s.where = "host" if kept else "none"
             self.stats.evictions += 1
+            freed += n_all
+        if freed < need:
+            raise RuntimeError("pool too small for this call even after evicting every other session")
 
     # ------------------------------------------------------------------ calls
     def run_group(self, calls: Sequence[Tuple[int, int, np.ndarray]]):
         """calls: (session id, call index, prompt tokens); distinct sessions.  Returns the match records."""
+        torch = self._torch
         B = self.shape.block_tokens
         self.clock += 1
         busy = {sid for sid, _, _ in calls}
@@ -177,6 +286,10 @@ class ReplayDriver:
             reuse = int(res[q]["reusable_tokens"]) // B
             if s.where == "device":
                 reuse = min(reuse, len(s.table))
+                self._truncate_host(s, reuse)
+                if s.event is not None:
+                    # blocks that are about to be rewritten may still be read by a checkpoint copy
+                    torch.cuda.current_stream().wait_event(s.event)
                 keep, drop = s.table[:reuse].copy(), s.table[reuse:]
                 self._release(drop)
                 s.table = keep
@@ -185,18 +298,21 @@ class ReplayDriver:
                 table = np.concatenate([keep, new]).astype(np.int32)
                 self.stats.device_hits += 1
             elif s.where == "host":
-                reuse = min(reuse, s.image_blocks)
+                reuse = min(reuse, s.host_blocks)
+                self._truncate_host(s, reuse)
                 self._make_room(need, busy)
                 table = self._alloc(need)
                 if reuse:
-                    n_img = s.image_blocks
-                    hl = tb.host_layout(wl.dense_strides(self.shape, n_img, self.order), n_img * self.shape.bytes_per_block)
-                    restores.append((table.copy(), 0, reuse, s.image, hl, sid, n_img))
+                    for e in s.extents:
+                        restores.append((table.copy(), e.first, e.n, e.image, e.hl))
+                    self.log.append(("restore", sid, table[:reuse].copy()))
+                    self.stats.restore_bytes += reuse * self.shape.bytes_per_block
                 self.stats.host_restores += 1
             else:
                 if s.last_use >= 0:
                     self.stats.capacity_misses += 1
                 reuse = 0
+                self._truncate_host(s, 0)
                 self._make_room(need, busy)
                 table = self._alloc(need)
                 self.stats.recomputes += 1
@@ -208,15 +324,11 @@ class ReplayDriver:
         # ---- restore the matched prefixes of all returning sessions in one call ----
         if restores:
             t0 = time.perf_counter()
-            self.ctx.kv_restore_batch(self.kv, [r[:5] for r in restores])
+            self.ctx.kv_restore_batch(self.kv, restores)
             self.ctx.sync()
             self.stats.restore_s += time.perf_counter() - t0
-            self.stats.restore_bytes += sum(r[2] for r in restores) * self.shape.bytes_per_block
-            for table, _, reuse, _, _, sid, n_img in restores:
-                self.log.append(("restore", sid, table[:reuse].copy(), n_img))
+        filled = []
         for s, k, toks, table, reuse, hashes in plans:
-            if s.where == "host":
-                self._drop_host(s)
             # ---- "prefill" of the unmatched tail: synthetic KV scattered into the new blocks ----
             m = len(table) - reuse
             if m:
@@ -228,4 +340,17 @@ class ReplayDriver:
                 self.log.append(("fill", s.sid, k, table[reuse:].copy()))
             s.table, s.where = table, "device"
             s.tokens, s.hashes, s.last_use = toks, hashes, self.clock
+            filled.append(s)
+        # ---- the call has finished: checkpoint its newly aligned blocks in the background ----
+        if self.checkpoint == "incremental":
+            fill_done = torch.cuda.Event()
+            fill_done.record()
+            for s in filled:
+                self._checkpoint(s, busy, fill_done)
         return res
+
+    def drain(self):
+        """Wait for every outstanding checkpoint copy (switch barrier, App. B)."""
+        self.ckpt_stream.synchronize()
+        for s in self.sessions.values():
+            s.event = None

@@ -1,6 +1,7 @@
 """GPU parity for the session-replay mix: 30 sessions with lognormal depth and prompt length,
 97 % high-reuse continuations, a pool capped at the block count of a 60 GB Qwen3-235B pool, LRU
-eviction to pinned host images and restore on return.  Every byte-moving step the driver logs is
+eviction, checkpoints of newly aligned blocks after every call (or whole-session copies at
+eviction) and restore on return.  Every byte-moving step the driver logs is
 replayed on the CPU oracle over a host mirror of the pool; pool, host images, match records and
 hashes must agree exactly.  The KV shape is cut to 2 layers x 2 heads x 64 (16 KiB per block) so
 the mirror stays small; block counts, tables and the schedule are those of the full shape.
@@ -34,8 +35,66 @@ def _groups(schedule, size):
     return out
 
 
-@pytest.mark.parametrize("order,host_budget_frac", [("PF", 0.35), ("LF", 10.0)])
-def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac):
+class Mirror:
+    """The oracle's copy of the driver's state: pool planes and, per session, checkpoint extents."""
+
+    def __init__(self, shape, planes, order):
+        self.shape, self.oshape = shape, orc.KvShape(shape.num_layers, shape.num_kv_heads, shape.block_tokens, shape.head_dim)
+        self.planes, self.order = planes, order
+        self.ext = {}                                   # sid -> list of [first, n, cap, image]
+
+    def apply(self, entry, calls, before, content):
+        shape, op = self.shape, entry[0]
+        if op == "match":
+            _, ids, got, hashes = entry
+            at = 0
+            for q, (sid, k) in enumerate(ids):
+                m, hc = orc.prefix_match(calls[q][2], before[sid], shape.block_tokens, wl.HASH_SEED)
+                assert (int(got[q]["lcp_tokens"]), int(got[q]["matched_blocks"]), int(got[q]["reusable_tokens"]),
+                        int(got[q]["hash_token_disagree"])) == (m.lcp_tokens, m.matched_blocks, m.reusable_tokens, 0)
+                assert np.array_equal(hashes[at:at + hc.size], hc)
+                at += hc.size
+        elif op == "checkpoint":
+            _, sid, first, ids = entry
+            img = np.zeros(ids.size * shape.bytes_per_block, np.uint8)
+            orc.kv_offload(self.oshape, self.planes, ids, 0, ids.size, img, wl.dense_strides(shape, ids.size, self.order))
+            exts = self.ext.setdefault(sid, [])
+            assert first == (exts[-1][0] + exts[-1][1] if exts else 0)          # extents are appended in order
+            exts.append([first, ids.size, ids.size, img])
+        elif op == "truncate":
+            _, sid, keep = entry
+            self.ext[sid] = [[f, min(n, keep - f), cap, img] for f, n, cap, img in self.ext.get(sid, []) if f < keep]
+        elif op in ("drop_host", "evict_lost"):
+            self.ext.pop(entry[1], None)
+        elif op == "evict":
+            pass
+        elif op == "restore":
+            _, sid, table = entry
+            covered = 0
+            for f, n, cap, img in self.ext[sid]:
+                orc.kv_restore(self.oshape, self.planes, table, f, n, img, wl.dense_strides(shape, cap, self.order))
+                covered += n
+            assert covered == table.size
+        elif op == "fill":
+            _, sid, k, ids = entry
+            img = content(sid, k, ids.size * shape.bytes_per_block)
+            orc.kv_restore(self.oshape, self.planes, ids, 0, ids.size, img, wl.dense_strides(shape, ids.size, "PF"))
+        else:
+            raise AssertionError(op)
+
+    def check_host_images(self, drv):
+        drv.drain()
+        for sid, s in drv.sessions.items():
+            mine = self.ext.get(sid, [])
+            assert [(e.first, e.n, e.cap) for e in s.extents] == [(f, n, cap) for f, n, cap, _ in mine], sid
+            for e, (_, _, _, img) in zip(s.extents, mine):
+                assert np.array_equal(e.image.numpy(), img), sid
+
+
+@pytest.mark.parametrize("order,host_budget_frac,checkpoint", [("PF", 0.35, "eviction"), ("LF", 10.0, "eviction"),
+                                                               ("PF", 10.0, "incremental"), ("LF", 10.0, "incremental"),
+                                                               ("PF", 0.9, "incremental")])
+def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac, checkpoint):
     shape = wl.KvShape(2, 2, 16, 64)
     full = wl.QWEN235
     pool_blocks = int(60e9) // full.bytes_per_block                       # 19,479 blocks, as at the full shape
@@ -45,18 +104,17 @@ def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac):
     planes_np = [g.integers(0, 256, size=pool_blocks * shape.chunk_bytes, dtype=np.uint8)
                  for _ in range(shape.num_layers * shape.num_planes)]
     d_planes = [torch.from_numpy(p).cuda() for p in planes_np]
-    mirror = [p.copy() for p in planes_np]
+    mirror = Mirror(shape, [p.copy() for p in planes_np], order)
     kv, keep = tb.kv_layout(shape, [t.data_ptr() for t in d_planes], pool_blocks)
-    oshape = orc.KvShape(shape.num_layers, shape.num_kv_heads, shape.block_tokens, shape.head_dim)
     total_kv = sum(shape.blocks_for(c.prompt_tokens) for c in schedule[:30]) * shape.bytes_per_block
     ctx = tb.Talaria(0, bounce_bytes=8 << 20, dma_min_bytes=4 << 20)      # both variants get exercised
     log = []
     drv = ReplayDriver(ctx, shape, kv, pool_blocks, int(total_kv * host_budget_frac), wl.HASH_SEED, _content,
                        lambda n: torch.empty(n, dtype=torch.uint8, pin_memory=True),
-                       lambda a: torch.from_numpy(a).cuda(), order=order, log=log)
-    streams, mirror_img, tg = {}, {}, wl.rng(4, 2)
+                       lambda a: torch.from_numpy(a).cuda(), order=order, log=log, checkpoint=checkpoint)
+    streams, tg = {}, wl.rng(4, 2)
     try:
-        for group in _groups(schedule, 4):
+        for gi, group in enumerate(_groups(schedule, 4)):
             calls = []
             for c in group:
                 prev = streams.get(c.session)
@@ -65,40 +123,15 @@ def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac):
                 calls.append((c.session, c.index, toks))
             before = {sid: streams.get(sid, np.zeros(0, np.int32)) for sid, _, _ in calls}
             log.clear()
-            res = drv.run_group(calls)
+            drv.run_group(calls)
             for entry in log:
-                op = entry[0]
-                if op == "match":
-                    _, ids, got, hashes = entry
-                    at = 0
-                    for q, (sid, k) in enumerate(ids):
-                        m, hc = orc.prefix_match(calls[q][2], before[sid], 16, wl.HASH_SEED)
-                        assert (int(got[q]["lcp_tokens"]), int(got[q]["matched_blocks"]), int(got[q]["reusable_tokens"]),
-                                int(got[q]["hash_token_disagree"])) == (m.lcp_tokens, m.matched_blocks, m.reusable_tokens, 0)
-                        assert np.array_equal(hashes[at:at + hc.size], hc)
-                        at += hc.size
-                elif op == "offload":
-                    _, sid, table = entry
-                    n = table.size
-                    img = np.zeros(n * shape.bytes_per_block, np.uint8)
-                    orc.kv_offload(oshape, mirror, table, 0, n, img, wl.dense_strides(shape, n, order))
-                    mirror_img[sid] = img
-                    s = drv.sessions[sid]
-                    if s.image is not None:
-                        assert np.array_equal(s.image.numpy(), img), sid
-                elif op == "drop_host":
-                    mirror_img.pop(entry[1], None)
-                elif op == "restore":
-                    _, sid, table, n_img = entry
-                    orc.kv_restore(oshape, mirror, table, 0, table.size, mirror_img[sid], wl.dense_strides(shape, n_img, order))
-                elif op == "fill":
-                    _, sid, k, ids = entry
-                    img = _content(sid, k, ids.size * shape.bytes_per_block)
-                    orc.kv_restore(oshape, mirror, ids, 0, ids.size, img, wl.dense_strides(shape, ids.size, "PF"))
+                mirror.apply(entry, calls, before, _content)
             for sid, _, toks in calls:
                 streams[sid] = toks
-                mirror_img.pop(sid, None) if drv.sessions[sid].where == "device" else None
-        for d, m in zip(d_planes, mirror):
+            if gi % 8 == 7:
+                mirror.check_host_images(drv)
+        mirror.check_host_images(drv)
+        for d, m in zip(d_planes, mirror.planes):
             assert np.array_equal(d.cpu().numpy(), m)
         # block ownership stays consistent: no block is owned twice or both owned and free
         owned = np.concatenate([s.table for s in drv.sessions.values() if s.where == "device"])
@@ -106,9 +139,15 @@ def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac):
         assert not set(owned.tolist()) & set(drv.free)
         assert owned.size + len(drv.free) == pool_blocks
         st = drv.stats
-        assert st.calls == len(schedule) and st.evictions > 0 and st.host_restores > 0
+        assert st.calls == len(schedule) and st.evictions > 0
         assert st.device_hits + st.host_restores + st.recomputes == st.calls
-        if host_budget_frac < 1:
-            assert st.capacity_misses > 0
+        if host_budget_frac >= 1:
+            assert st.host_restores > 0 and st.capacity_misses == 0
+        if checkpoint == "eviction" and host_budget_frac < 1:
+            assert st.capacity_misses > 0 and st.host_restores > 0
+        if checkpoint == "incremental":
+            # the barrier at eviction found most of the session on the host already
+            assert st.checkpoint_bytes > 0
+            assert st.evict_bytes_already_on_host > 10 * st.evict_bytes_copied
     finally:
         ctx.destroy()
