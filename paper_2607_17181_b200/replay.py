@@ -99,16 +99,20 @@ class ReplayDriver:
     def __init__(self, ctx: tb.Talaria, shape: wl.KvShape, kv, pool_blocks: int, host_budget_bytes: int,
                  seed: int, content: Callable[[int, int, int], np.ndarray], alloc_pinned: Callable[[int], object],
                  to_device: Callable[[np.ndarray], object], order: str = "PF", log: Optional[list] = None,
-                 free_pinned: Optional[Callable[[object], None]] = None, checkpoint: str = "incremental"):
+                 free_pinned: Optional[Callable[[object], None]] = None, checkpoint: str = "incremental",
+                 max_extent_blocks: int = 512):
         """content(session, call_index, nbytes) -> uint8 array: the synthetic KV of a call's new blocks.
         alloc_pinned(nbytes) -> pinned host tensor; free_pinned(tensor) gives it back (optional);
         to_device(array) -> device tensor (memory plumbing).
-        checkpoint: "incremental" (after every call, asynchronously) or "eviction" (whole session when evicted)."""
+        checkpoint: "incremental" (after every call, asynchronously) or "eviction" (whole session when evicted).
+        max_extent_blocks: a checkpoint is cut into host images of at most this many blocks, so the
+        pinned allocator is never asked for one multi-gigabyte piece."""
         import torch
         assert checkpoint in ("incremental", "eviction")
         self.ctx, self.shape, self.kv = ctx, shape, kv
         self.pool_blocks, self.host_budget = pool_blocks, host_budget_bytes
         self.seed, self.order, self.checkpoint = seed, order, checkpoint
+        self.max_extent_blocks = max(1, max_extent_blocks)
         self.content, self.alloc_pinned, self.to_device = content, alloc_pinned, to_device
         self.free_pinned = free_pinned
         self.free: List[int] = list(range(pool_blocks))      # min-heap: low addresses are reused first
@@ -177,14 +181,28 @@ class ReplayDriver:
             self.log.append(("drop_host", old[0].sid))
         return True
 
-    def _new_extent(self, s: SessionState, first: int, n: int) -> Extent:
-        nbytes = n * self.shape.bytes_per_block
-        image = self.alloc_pinned(nbytes)
-        hl = tb.host_layout(wl.dense_strides(self.shape, n, self.order), nbytes)
-        e = Extent(first, n, image, hl, n)
-        self.host_bytes += nbytes
-        s.extents.append(e)
-        return e
+    def _offload_range(self, s: SessionState, first: int, n: int, busy: set, stream=None) -> int:
+        """Copy blocks [first, first + n) of a resident session to new host extents of bounded size.
+        Returns the number of blocks that found room on the host (a prefix of the range)."""
+        done = 0
+        while done < n:
+            m = min(self.max_extent_blocks, n - done)
+            nbytes = m * self.shape.bytes_per_block
+            if not self._host_room(nbytes, busy | {s.sid}):
+                break
+            try:
+                image = self.alloc_pinned(nbytes)
+            except MemoryError:                       # the pinned allocator is fragmented: same as no room
+                break
+            hl = tb.host_layout(wl.dense_strides(self.shape, m, self.order), nbytes)
+            e = Extent(first + done, m, image, hl, m)
+            self.host_bytes += nbytes
+            s.extents.append(e)
+            self.ctx.kv_offload(self.kv, s.table, e.first, m, e.image, e.hl, stream=stream)
+            self.stats.offload_bytes += nbytes
+            self.log.append(("checkpoint", s.sid, e.first, s.table[e.first:e.first + m].copy()))
+            done += m
+        return done
 
     def _checkpoint(self, s: SessionState, busy: set, fill_done):
         """Asynchronously checkpoint the session's newly aligned (full) blocks."""
@@ -193,17 +211,14 @@ class ReplayDriver:
         n = full - first
         if n <= 0:
             return
-        if not self._host_room(n * self.shape.bytes_per_block, busy | {s.sid}):
-            self.stats.checkpoints_skipped += 1
-            return
-        e = self._new_extent(s, first, n)
         self.ckpt_stream.wait_event(fill_done)
-        self.ctx.kv_offload(self.kv, s.table, first, n, e.image, e.hl, stream=self.ckpt_stream)
-        s.event = self._torch.cuda.Event()
-        s.event.record(self.ckpt_stream)
-        self.stats.checkpoint_bytes += n * self.shape.bytes_per_block
-        self.stats.offload_bytes += n * self.shape.bytes_per_block
-        self.log.append(("checkpoint", s.sid, first, s.table[first:first + n].copy()))
+        done = self._offload_range(s, first, n, busy, stream=self.ckpt_stream)
+        if done < n:
+            self.stats.checkpoints_skipped += 1
+        if done:
+            s.event = self._torch.cuda.Event()
+            s.event.record(self.ckpt_stream)
+            self.stats.checkpoint_bytes += done * self.shape.bytes_per_block
 
     # --------------------------------------------------------------- eviction
     def _make_room(self, need: int, busy: set):
@@ -222,14 +237,9 @@ class ReplayDriver:
             rest = n_all - first                                  # not on the host yet (normally the tail block)
             kept = True
             if rest > 0:
-                if self._host_room(rest * self.shape.bytes_per_block, busy | {s.sid}):
-                    e = self._new_extent(s, first, rest)
-                    self.ctx.kv_offload(self.kv, s.table, first, rest, e.image, e.hl)
-                    self.stats.offload_bytes += rest * self.shape.bytes_per_block
-                    self.stats.evict_bytes_copied += rest * self.shape.bytes_per_block
-                    self.log.append(("checkpoint", s.sid, first, s.table[first:first + rest].copy()))
-                else:
-                    kept = False                                  # no host room: this session's KV is lost
+                done = self._offload_range(s, first, rest, busy)
+                self.stats.evict_bytes_copied += done * self.shape.bytes_per_block
+                kept = done == rest                               # no host room: this session's KV is lost
             # switch barrier for this session: its checkpoint copies and the tail copy are done
             if s.event is not None:
                 s.event.synchronize()
