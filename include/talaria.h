@@ -407,6 +407,79 @@ talaria_status_t talaria_prestage(talaria_ctx *ctx, const talaria_copy_t *plan, 
 int64_t talaria_mark_dirty(const talaria_copy_t *plan, int64_t n, const void *alloc_base,
                            int64_t alloc_bytes, const uint8_t *staged_bitmap, uint8_t *dirty_bitmap);
 
+/* ---- stable-address HBM layout (Sec. 4.2, Sec. 4.4) -------------------------------- */
+
+/* One managed region for every model of a cold-pool instance (Sec. 4.2): for the active model
+ * the weights grow up from the low-address end, the runtime buffers are anchored at the
+ * high-address end, and the gap between them is the paged KV pool.  Pure host arithmetic:
+ * region_base is a DEVICE address that is only ever added to, never dereferenced.
+ *
+ * Layout of model m in a region of S bytes (A = align, a power of two; C = chunk_bytes, a
+ * multiple of A; LP = num_layers*num_planes):
+ *     weights  [0, weight_bytes)
+ *     runtime  [R, R + runtime_bytes)          R = floor((S - runtime_bytes) / A) * A
+ *     KV pool  plane k = [K + k*NB*C, +NB*C)   K = ceil(weight_bytes / A) * A,
+ *                                              NB = floor((R - K) / (LP*C)) >= 1 (else EXTENT)
+ * Every address is a function of (region, model) only: a model finds its weights, KV planes and
+ * runtime buffers where they were the last time (the restore-time pointer check of Sec. 4.2
+ * compares exactly these bases).
+ *
+ * activate(m)    : m becomes the active model; all of its NB blocks are free; any staging
+ *                  placement is forgotten (the switch consumed it).
+ * alloc_blocks   : n block ids, lowest free ids first (Sec. 4.4: low addresses are reused first,
+ *                  which keeps the plane tails clean), passing over rows under an active staging
+ *                  write.  A block id is a row of EVERY plane; for each staged chunk (bit set in
+ *                  staged_bitmap, or every placed chunk if that is NULL) that loses a row to the
+ *                  allocation, its bit in dirty_bitmap (nullable, in/out) is set; *n_dirtied
+ *                  (nullable) counts bits that changed.  NO_MEMORY if fewer than n ids are
+ *                  available (nothing is taken).
+ * free_blocks    : INVALID_ARG for an id that is out of range, already free or given twice.
+ * stage_place    : plans pre-staging of model `next` (Sec. 4.4): its weights are cut into chunks
+ *                  of chunk_bytes (the last may be short); chunk j goes to the next usable tail
+ *                  slot, slots being taken tail slot by tail slot across all planes (slot t of a
+ *                  plane = rows [NB-(t+1)*r, NB-t*r), r = ceil(chunk_bytes / C)).  A slot is
+ *                  usable when all its rows are free and unlocked and none of its bytes lies in
+ *                  [0, ceil(next.weight_bytes / A) * A), where the switch will write.  plan_out[j]
+ *                  (HOST array, capacity >= *n_chunks_out, else EXTENT) = { src_dev = the slot's
+ *                  address or NULL if no slot was left, src_host = host_weights + j*chunk_bytes
+ *                  (NULL when host_weights is NULL), dst_dev = next's weights base + j*chunk_bytes,
+ *                  bytes, chunk_id = j }: ready for talaria_prestage, talaria_mark_dirty and
+ *                  talaria_stage / talaria_stage_plan_create.
+ * lock_chunk     : marks a placed chunk as being written (locked != 0) or done (0).
+ * staging_slack  : bytes of weights that could still be staged for `next` at this chunk size
+ *                  (usable slots not holding a chunk, times chunk_bytes): the paper's staging
+ *                  slack signal. */
+typedef struct talaria_bump talaria_bump;
+typedef struct {
+  int64_t weight_bytes, runtime_bytes;
+  int32_t num_layers, num_planes;
+  int64_t chunk_bytes;
+} talaria_model_desc_t;
+typedef struct {
+  void *weights_base;
+  int64_t weights_bytes;
+  void *kv_base;
+  int64_t kv_bytes;          /* num_layers * num_planes * num_blocks * chunk_bytes */
+  void *runtime_base;
+  int64_t runtime_bytes;
+  int64_t num_blocks;        /* rows per plane = pool capacity in blocks */
+} talaria_bump_view_t;
+talaria_status_t talaria_bump_create(talaria_bump **out, void *region_base, int64_t region_bytes, int64_t align,
+                                     const talaria_model_desc_t *models, int32_t n_models);
+talaria_status_t talaria_bump_destroy(talaria_bump *b);
+/* plane_base_out: HOST array [num_layers*num_planes] or NULL; usable as talaria_kv_layout_t.plane_base. */
+talaria_status_t talaria_bump_view(talaria_bump *b, int32_t model, talaria_bump_view_t *view, void **plane_base_out);
+talaria_status_t talaria_bump_activate(talaria_bump *b, int32_t model, talaria_bump_view_t *view /*nullable*/);
+talaria_status_t talaria_bump_alloc_blocks(talaria_bump *b, int64_t n, int32_t *ids_out, const uint8_t *staged_bitmap,
+                                           uint8_t *dirty_bitmap, int64_t *n_dirtied);
+talaria_status_t talaria_bump_free_blocks(talaria_bump *b, const int32_t *ids, int64_t n);
+int64_t talaria_bump_free_count(talaria_bump *b);
+talaria_status_t talaria_bump_stage_place(talaria_bump *b, int32_t next_model, int64_t chunk_bytes,
+                                          const void *host_weights, talaria_copy_t *plan_out, int64_t plan_capacity,
+                                          int64_t *n_chunks_out, int64_t *n_placed_out /*nullable*/);
+talaria_status_t talaria_bump_lock_chunk(talaria_bump *b, int32_t chunk_id, int32_t locked);
+int64_t talaria_bump_staging_slack(talaria_bump *b, int32_t next_model, int64_t chunk_bytes);
+
 /* ---- argument checks that need no GPU ------------------------------------------ */
 
 /* The same host-side validation the copy and stage calls apply, callable on its own

@@ -5,7 +5,9 @@ benchmark's CPU-baseline leg.  It never touches CUDA, never imports the CUDA
 package, and the CUDA package never imports it.
 
 Every function takes and returns numpy arrays (host memory).  The arithmetic
-lives in the C file; this module only marshals arguments.
+lives in the C file; this module only marshals arguments -- except for the two
+pieces of host bookkeeping at the end (page registry, stable-address layout),
+whose definitions are written out directly with dicts, sets and loops.
 """
 from __future__ import annotations
 
@@ -358,3 +360,120 @@ class Registry:
 
     def __len__(self):
         return len(self.d)
+
+
+# ------------------------------------------------------- stable-address layout
+
+
+class BumpLayout:
+    """Plain definition of the stable-address HBM layout (Sec. 4.2) and its staging surface
+    (Sec. 4.4), written out with Python sets and loops; offsets are relative to the region base.
+
+    Layout of a model (weights up from the low end, runtime buffers anchored high, the gap is
+    the KV pool of LP planes x NB rows of C bytes):
+        weights [0, W);  runtime [R, R + Rt) with R = floor((S - Rt) / A) * A;
+        K = ceil(W / A) * A;  NB = floor((R - K) / (LP * C));  plane k = [K + k*NB*C, +NB*C).
+    Block ids are allocated lowest first, skipping rows under an active staging write; an
+    allocated id is a row of every plane and dirties each staged chunk that owns that row.
+    Staging for model `nxt`: chunk j takes the next usable tail slot, slots enumerated tail
+    slot by tail slot across planes; slot t of a plane = rows [NB-(t+1)r, NB-t*r) with
+    r = ceil(chunk / C); usable = all rows free and unlocked, and no byte below ceil(W_nxt/A)*A."""
+
+    def __init__(self, region_bytes: int, align: int, models):
+        """models: list of (weight_bytes, runtime_bytes, num_layers, num_planes, chunk_bytes)."""
+        self.S, self.A, self.models = region_bytes, align, [tuple(m) for m in models]
+        self.active = None
+
+    def view(self, m: int):
+        W, Rt, L, P, Cb = self.models[m]
+        A = self.A
+        K = -(-W // A) * A
+        R = (self.S - Rt) // A * A
+        NB = (R - K) // (L * P * Cb) if R >= K else 0
+        if NB < 1:
+            raise ValueError("region too small for this model")
+        return {"weights": (0, W), "runtime": (R, Rt), "kv": (K, L * P * NB * Cb), "num_blocks": NB,
+                "planes": [K + k * NB * Cb for k in range(L * P)]}
+
+    def activate(self, m: int):
+        self.active = m
+        self.NB = self.view(m)["num_blocks"]
+        self.free = set(range(self.NB))
+        self.chunks = []            # per chunk: None or (plane, row0)
+        self.locked = set()
+        self.r = 0
+
+    def _locked_rows(self):
+        rows = set()
+        for c in self.locked:
+            if self.chunks[c] is not None:
+                rows.update(range(self.chunks[c][1], self.chunks[c][1] + self.r))
+        return rows
+
+    def alloc_blocks(self, n: int, staged=None, dirty=None):
+        """Returns (ids, newly dirtied chunk ids).  staged / dirty: Python sets of chunk ids."""
+        avail = sorted(self.free - self._locked_rows())
+        if len(avail) < n:
+            raise MemoryError("not enough free blocks")
+        ids = avail[:n]
+        newly = []
+        for b in ids:
+            self.free.discard(b)
+            for c, place in enumerate(self.chunks):
+                if place is None or dirty is None:
+                    continue
+                if place[1] <= b < place[1] + self.r and (staged is None or c in staged) and c not in dirty:
+                    dirty.add(c)
+                    newly.append(c)
+        return ids, newly
+
+    def free_blocks(self, ids):
+        ids = list(ids)
+        if len(set(ids)) != len(ids) or any(b < 0 or b >= self.NB or b in self.free for b in ids):
+            raise ValueError("bad id in free_blocks")
+        self.free.update(ids)
+
+    def _usable_slots(self, nxt: int, chunk_bytes: int, taken=()):
+        W2 = self.models[nxt][0]
+        lim = -(-W2 // self.A) * self.A
+        _, _, L, P, Cb = self.models[self.active]
+        planes = self.view(self.active)["planes"]
+        r = -(-chunk_bytes // Cb)
+        blocked = self._locked_rows()
+        out = []
+        for t in range(self.NB // r):
+            row0 = self.NB - (t + 1) * r
+            rows = range(row0, row0 + r)
+            for k in range(L * P):
+                if (k, row0) in taken:
+                    continue
+                if planes[k] + row0 * Cb < lim:
+                    continue
+                if all(x in self.free and x not in blocked for x in rows):
+                    out.append((k, row0))
+        return out, r
+
+    def stage_place(self, nxt: int, chunk_bytes: int):
+        """Returns the plan: per chunk (staging offset or None, weights offset, nbytes)."""
+        W2 = self.models[nxt][0]
+        n_chunks = -(-W2 // chunk_bytes)
+        self.chunks, self.locked = [], set()
+        slots, self.r = self._usable_slots(nxt, chunk_bytes)
+        planes = self.view(self.active)["planes"]
+        Cb = self.models[self.active][4]
+        plan = []
+        for j in range(n_chunks):
+            place = slots[j] if j < len(slots) else None
+            self.chunks.append(place)
+            nbytes = min(chunk_bytes, W2 - j * chunk_bytes)
+            plan.append((None if place is None else planes[place[0]] + place[1] * Cb, j * chunk_bytes, nbytes))
+        return plan
+
+    def staging_slack(self, nxt: int, chunk_bytes: int) -> int:
+        Cb = self.models[self.active][4]
+        same = self.r == -(-chunk_bytes // Cb)
+        taken = {p for p in self.chunks if p is not None} if same else set()
+        saved = self.r
+        slots, _ = self._usable_slots(nxt, chunk_bytes, taken)
+        self.r = saved
+        return len(slots) * chunk_bytes

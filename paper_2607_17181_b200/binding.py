@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 _INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB_PATH = os.path.join(_HERE, "libtalaria.so")
-SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "prefix_pair.cu", "stage.cu", "registry.cu"]
+SOURCES = ["ctx.cu", "kv_copy.cu", "prefix.cu", "prefix_pair.cu", "stage.cu", "registry.cu", "bump.cu"]
 HEADERS = ["internal.h", "prefix_common.cuh"]
 
 OK = 0
@@ -90,6 +90,17 @@ class Counters(C.Structure):
                 ("last_variant", C.c_int32), ("reserved", C.c_int32)]
 
 
+class ModelDesc(C.Structure):
+    _fields_ = [("weight_bytes", C.c_int64), ("runtime_bytes", C.c_int64), ("num_layers", C.c_int32),
+                ("num_planes", C.c_int32), ("chunk_bytes", C.c_int64)]
+
+
+class BumpView(C.Structure):
+    _fields_ = [("weights_base", C.c_void_p), ("weights_bytes", C.c_int64), ("kv_base", C.c_void_p),
+                ("kv_bytes", C.c_int64), ("runtime_base", C.c_void_p), ("runtime_bytes", C.c_int64),
+                ("num_blocks", C.c_int64)]
+
+
 class KvXfer(C.Structure):
     _fields_ = [("block_table", C.c_void_p), ("first_block", C.c_int64), ("n_blocks", C.c_int64),
                 ("host", C.c_void_p), ("hl", HostLayout)]
@@ -127,6 +138,17 @@ _SIGNATURES = {
     "talaria_stage_plan_destroy": (C.c_int32, [_P, _P]),
     "talaria_prestage": (C.c_int32, [_P, _P, C.c_int64, _P, _P, _P, C.POINTER(StageStats), _P]),
     "talaria_mark_dirty": (C.c_int64, [_P, C.c_int64, _P, C.c_int64, _P, _P]),
+    "talaria_bump_create": (C.c_int32, [C.POINTER(_P), _P, C.c_int64, C.c_int64, C.POINTER(ModelDesc), C.c_int32]),
+    "talaria_bump_destroy": (C.c_int32, [_P]),
+    "talaria_bump_view": (C.c_int32, [_P, C.c_int32, C.POINTER(BumpView), _P]),
+    "talaria_bump_activate": (C.c_int32, [_P, C.c_int32, C.POINTER(BumpView)]),
+    "talaria_bump_alloc_blocks": (C.c_int32, [_P, C.c_int64, _P, _P, _P, C.POINTER(C.c_int64)]),
+    "talaria_bump_free_blocks": (C.c_int32, [_P, _P, C.c_int64]),
+    "talaria_bump_free_count": (C.c_int64, [_P]),
+    "talaria_bump_stage_place": (C.c_int32, [_P, C.c_int32, C.c_int64, _P, _P, C.c_int64, C.POINTER(C.c_int64),
+                                             C.POINTER(C.c_int64)]),
+    "talaria_bump_lock_chunk": (C.c_int32, [_P, C.c_int32, C.c_int32]),
+    "talaria_bump_staging_slack": (C.c_int64, [_P, C.c_int32, C.c_int64]),
     "talaria_check_block_table": (C.c_int32, [_P, C.c_int64, C.c_int64, C.c_int32]),
     "talaria_check_image_layout": (C.c_int32, [C.POINTER(KvLayout), C.c_int64, C.POINTER(HostLayout), C.POINTER(C.c_int64)]),
     "talaria_check_stage_plan": (C.c_int32, [_P, C.c_int64, _P, C.POINTER(StageStats)]),
@@ -268,6 +290,79 @@ class Registry:
     def destroy(self):
         if self._h:
             lib().talaria_registry_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class Bump:
+    """Stable-address layout of one managed HBM region (host arithmetic; needs no GPU).
+    models: sequence of (weight_bytes, runtime_bytes, num_layers, num_planes, chunk_bytes)."""
+
+    def __init__(self, region_base: int, region_bytes: int, models, align: int = 256):
+        self._h = C.c_void_p()
+        self.models = [ModelDesc(*m) for m in models]
+        arr = (ModelDesc * len(self.models))(*self.models)
+        rc = lib().talaria_bump_create(C.byref(self._h), region_base, region_bytes, align, arr, len(self.models))
+        if rc != OK:
+            self._h = C.c_void_p()
+            raise TalariaError(rc, "talaria_bump_create")
+
+    def _check(self, rc, what):
+        if rc != OK:
+            raise TalariaError(rc, what)
+
+    def view(self, model: int):
+        """(BumpView, list of plane base addresses) of a model: the same every time."""
+        v = BumpView()
+        d = self.models[model]
+        planes = (C.c_void_p * (d.num_layers * d.num_planes))()
+        self._check(lib().talaria_bump_view(self._h, model, C.byref(v), planes), "talaria_bump_view")
+        return v, [int(p or 0) for p in planes]
+
+    def activate(self, model: int) -> BumpView:
+        v = BumpView()
+        self._check(lib().talaria_bump_activate(self._h, model, C.byref(v)), "talaria_bump_activate")
+        return v
+
+    def alloc_blocks(self, n: int, staged_bitmap=None, dirty_bitmap=None):
+        """(ids, number of chunks newly marked dirty); dirty_bitmap is updated in place."""
+        ids = np.zeros(max(n, 1), np.int32)
+        nd = C.c_int64()
+        self._check(lib().talaria_bump_alloc_blocks(self._h, n, _ptr(ids), _ptr(staged_bitmap), _ptr(dirty_bitmap),
+                                                    C.byref(nd)), "talaria_bump_alloc_blocks")
+        return ids[:n], nd.value
+
+    def free_blocks(self, ids):
+        ids = _i32(ids)
+        self._check(lib().talaria_bump_free_blocks(self._h, _ptr(ids), ids.size), "talaria_bump_free_blocks")
+
+    def free_count(self) -> int:
+        return int(lib().talaria_bump_free_count(self._h))
+
+    def stage_place(self, next_model: int, chunk_bytes: int, host_weights: int = 0):
+        """(plan as COPY_DTYPE array, chunks that found a staging slot)."""
+        d = self.models[next_model]
+        cap = max(1, -(-d.weight_bytes // chunk_bytes))
+        plan = np.zeros(cap, COPY_DTYPE)
+        n, placed = C.c_int64(), C.c_int64()
+        self._check(lib().talaria_bump_stage_place(self._h, next_model, chunk_bytes, host_weights or None, _ptr(plan),
+                                                   cap, C.byref(n), C.byref(placed)), "talaria_bump_stage_place")
+        return plan[:n.value], placed.value
+
+    def lock_chunk(self, chunk_id: int, locked: bool):
+        self._check(lib().talaria_bump_lock_chunk(self._h, chunk_id, 1 if locked else 0), "talaria_bump_lock_chunk")
+
+    def staging_slack(self, next_model: int, chunk_bytes: int) -> int:
+        return int(lib().talaria_bump_staging_slack(self._h, next_model, chunk_bytes))
+
+    def destroy(self):
+        if self._h:
+            lib().talaria_bump_destroy(self._h)
             self._h = C.c_void_p()
 
     def __del__(self):
