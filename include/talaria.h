@@ -131,6 +131,18 @@ typedef struct {
   int64_t d2d_bytes, h2d_bytes, dirty_chunks, missing_chunks;
 } talaria_stage_stats_t;
 
+/* App. D "Path classification" also records the D2D and H2D gather times of a switch, and the
+ * router charges a measured restore cost (Sec. 3.3): optional per-call timing from CUDA events
+ * on the streams the work runs on.  op: 1 offload, 2 restore, 3 stage; the leg fields that do
+ * not apply are 0.  For a stage, d2d_ms is the gather kernel and h2d_ms the host reloads, which
+ * overlap, so total_ms is less than their sum. */
+typedef struct {
+  float total_ms;           /* from the call's first to its last piece of work on `stream`   */
+  float d2d_ms, h2d_ms, d2h_ms;
+  int32_t op;
+  int32_t reserved;
+} talaria_timing_t;
+
 typedef struct {
   int64_t kernel_launches;  /* kernels of this library launched since create / reset         */
   int64_t memcpy_calls;     /* copy-engine copies enqueued (payload and descriptors)         */
@@ -224,7 +236,8 @@ talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
  * that first call before any stream capture.  All calls in a process share the one
  * scratch array per device: two calls whose kernels can overlap on the GPU
  * (different streams, no ordering between them) race on it and must be serialised
- * by the caller.  The array keeps the previous call's contents; nothing in it
+ * by the caller.  Host threads may call concurrently: the two launches of a call are
+ * issued under one internal lock.  The array keeps the previous call's contents; nothing in it
  * needs clearing because every word that is read is written first in the same
  * call. */
 talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const int32_t *d_cont_tokens,
@@ -514,6 +527,11 @@ const char *talaria_strerror(talaria_status_t status);
 /* cudaError_t value of the last failed CUDA call in this context (0 if none). */
 int32_t talaria_last_cuda_error(talaria_ctx *ctx);
 talaria_status_t talaria_get_counters(talaria_ctx *ctx, talaria_counters_t *out);
+/* Timing is off by default (events cost a little on every call).  With it on, every offload,
+ * restore (all forms) and stage records its events; talaria_get_timing waits for the last timed
+ * call to finish and returns its times (INVALID_ARG if no call was timed yet). */
+talaria_status_t talaria_set_timing(talaria_ctx *ctx, int32_t enabled);
+talaria_status_t talaria_get_timing(talaria_ctx *ctx, talaria_timing_t *out);
 talaria_status_t talaria_reset_counters(talaria_ctx *ctx);
 
 #ifdef __cplusplus

@@ -101,6 +101,11 @@ class BumpView(C.Structure):
                 ("num_blocks", C.c_int64)]
 
 
+class Timing(C.Structure):
+    _fields_ = [("total_ms", C.c_float), ("d2d_ms", C.c_float), ("h2d_ms", C.c_float), ("d2h_ms", C.c_float),
+                ("op", C.c_int32), ("reserved", C.c_int32)]
+
+
 class KvXfer(C.Structure):
     _fields_ = [("block_table", C.c_void_p), ("first_block", C.c_int64), ("n_blocks", C.c_int64),
                 ("host", C.c_void_p), ("hl", HostLayout)]
@@ -157,6 +162,8 @@ _SIGNATURES = {
     "talaria_last_cuda_error": (C.c_int32, [_P]),
     "talaria_get_counters": (C.c_int32, [_P, C.POINTER(Counters)]),
     "talaria_reset_counters": (C.c_int32, [_P]),
+    "talaria_set_timing": (C.c_int32, [_P, C.c_int32]),
+    "talaria_get_timing": (C.c_int32, [_P, C.POINTER(Timing)]),
 }
 
 _lib = None
@@ -558,6 +565,15 @@ class Talaria:
         c = Counters()
         self._check(lib().talaria_get_counters(self._h, C.byref(c)), "talaria_get_counters")
         return c
+
+    def set_timing(self, enabled: bool):
+        self._check(lib().talaria_set_timing(self._h, 1 if enabled else 0), "talaria_set_timing")
+
+    def get_timing(self) -> Timing:
+        """Times of the last timed offload / restore / stage (waits for it to finish)."""
+        t = Timing()
+        self._check(lib().talaria_get_timing(self._h, C.byref(t)), "talaria_get_timing")
+        return t
 
     def reset_counters(self):
         self._check(lib().talaria_reset_counters(self._h), "talaria_reset_counters")

@@ -206,6 +206,8 @@ static void destroy_impl(talaria_ctx *ctx) {
     cudaStreamSynchronize(ctx->reload_stream);
     cudaStreamDestroy(ctx->reload_stream);
   }
+  for (cudaEvent_t e : ctx->tm)
+    if (e) cudaEventDestroy(e);
   if (ctx->reload_fork) cudaEventDestroy(ctx->reload_fork);
   if (ctx->reload_done) cudaEventDestroy(ctx->reload_done);
   for (auto &s : ctx->ring) {
@@ -277,6 +279,7 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
     int prio_least = 0, prio_greatest = 0;
     TAL_CUDA(ctx, cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
     TAL_CUDA(ctx, cudaStreamCreateWithPriority(&ctx->reload_stream, cudaStreamNonBlocking, prio_least));
+    for (cudaEvent_t &e : ctx->tm) TAL_CUDA(ctx, cudaEventCreate(&e));
     TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->reload_fork, cudaEventDisableTiming));
     TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->reload_done, cudaEventDisableTiming));
     for (auto &ln : ctx->lane) {
@@ -369,6 +372,36 @@ extern "C" talaria_status_t talaria_get_counters(talaria_ctx *ctx, talaria_count
   if (!ctx || !out) return TALARIA_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lk(ctx->mu);
   *out = ctx->counters;
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_set_timing(talaria_ctx *ctx, int32_t enabled) {
+  if (!ctx) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  ctx->timing = enabled != 0;
+  return TALARIA_OK;
+}
+
+extern "C" talaria_status_t talaria_get_timing(talaria_ctx *ctx, talaria_timing_t *out) {
+  if (!ctx || !out) return TALARIA_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lk(ctx->mu);
+  DeviceGuard g(ctx->device);
+  if (ctx->tm_op == 0) return TALARIA_ERR_INVALID_ARG;
+  talaria_timing_t t{};
+  t.op = ctx->tm_op;
+  TAL_CUDA(ctx, cudaEventSynchronize(ctx->tm[1]));
+  TAL_CUDA(ctx, cudaEventElapsedTime(&t.total_ms, ctx->tm[0], ctx->tm[1]));
+  if (ctx->tm_d2d) {
+    TAL_CUDA(ctx, cudaEventSynchronize(ctx->tm[3]));
+    TAL_CUDA(ctx, cudaEventElapsedTime(&t.d2d_ms, ctx->tm[2], ctx->tm[3]));
+  }
+  if (ctx->tm_h2d) {
+    TAL_CUDA(ctx, cudaEventSynchronize(ctx->tm[5]));
+    TAL_CUDA(ctx, cudaEventElapsedTime(&t.h2d_ms, ctx->tm[4], ctx->tm[5]));
+  }
+  if (t.op == 1) t.d2h_ms = t.total_ms;
+  if (t.op == 2) t.h2d_ms = t.total_ms;
+  *out = t;
   return TALARIA_OK;
 }
 

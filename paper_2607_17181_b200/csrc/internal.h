@@ -78,6 +78,12 @@ struct talaria_ctx {
   unsigned int *status_dev = nullptr;   // the same word as the device sees it
   int32_t last_cuda_error = 0;
   talaria_counters_t counters{};
+  // optional per-call timing: [0],[1] whole call on the caller's stream; [2],[3] the D2D gather
+  // kernel of a stage; [4],[5] its host reloads on the reload stream
+  bool timing = false;
+  cudaEvent_t tm[6] = {};
+  int32_t tm_op = 0;                  // 0 = nothing timed yet
+  bool tm_d2d = false, tm_h2d = false;
 };
 
 namespace tal {
@@ -96,6 +102,21 @@ talaria_status_t cuda_fail(talaria_ctx *ctx, cudaError_t e);
     talaria_status_t s__ = (expr);                            \
     if (s__ != TALARIA_OK) return s__;                        \
   } while (0)
+
+// Brackets one timed call on the caller's stream (no-op while timing is off).
+struct CallTimer {
+  talaria_ctx *ctx;
+  cudaStream_t stream;
+  CallTimer(talaria_ctx *c, cudaStream_t s, int32_t op) : ctx(c), stream(s) {
+    if (!ctx->timing) return;
+    ctx->tm_op = op;
+    ctx->tm_d2d = ctx->tm_h2d = false;
+    cudaEventRecord(ctx->tm[0], stream);
+  }
+  ~CallTimer() {
+    if (ctx->timing) cudaEventRecord(ctx->tm[1], stream);
+  }
+};
 
 // RAII: make the context's device current for the duration of a call.
 struct DeviceGuard {

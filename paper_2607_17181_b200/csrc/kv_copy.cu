@@ -791,6 +791,7 @@ extern "C" talaria_status_t talaria_kv_offload(talaria_ctx *ctx, const talaria_k
                                                int64_t n_blocks, void *host_dst,
                                                const talaria_host_layout_t *hl, void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 1);
   return kv_transfer(ctx, kv, block_table, first_block, n_blocks, host_dst, hl, (cudaStream_t)stream, true, false);
 }
 
@@ -799,6 +800,7 @@ extern "C" talaria_status_t talaria_kv_restore(talaria_ctx *ctx, const talaria_k
                                                int64_t n_blocks, const void *host_src,
                                                const talaria_host_layout_t *hl, void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 2);
   return kv_transfer(ctx, kv, new_block_table, first_block, n_blocks, (void *)host_src, hl,
                      (cudaStream_t)stream, false, false);
 }
@@ -809,6 +811,7 @@ extern "C" talaria_status_t talaria_kv_restore_layered(talaria_ctx *ctx, const t
                                                        const talaria_host_layout_t *hl,
                                                        void *const *layer_events, void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 2);
   return kv_restore_layered(ctx, kv, new_block_table, first_block, n_blocks, host_src, hl, layer_events,
                             (cudaStream_t)stream);
 }
@@ -818,6 +821,7 @@ extern "C" talaria_status_t talaria_kv_offload_pages(talaria_ctx *ctx, const tal
                                                      int64_t n_blocks, void *host_pool, int64_t pool_bytes,
                                                      const int64_t *page_offsets, void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 1);
   return kv_transfer_pages(ctx, kv, block_table, first_block, n_blocks, host_pool, pool_bytes, page_offsets,
                            (cudaStream_t)stream, true);
 }
@@ -827,6 +831,7 @@ extern "C" talaria_status_t talaria_kv_restore_pages(talaria_ctx *ctx, const tal
                                                      int64_t n_blocks, const void *host_pool, int64_t pool_bytes,
                                                      const int64_t *page_offsets, void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 2);
   return kv_transfer_pages(ctx, kv, new_block_table, first_block, n_blocks, (void *)host_pool, pool_bytes,
                            page_offsets, (cudaStream_t)stream, false);
 }
@@ -973,6 +978,7 @@ extern "C" talaria_status_t talaria_kv_offload_batch(talaria_ctx *ctx, const tal
                                                      const talaria_kv_xfer_t *xfers, int32_t n_xfers,
                                                      void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 1);
   return kv_batch(ctx, kv, xfers, n_xfers, (cudaStream_t)stream, true);
 }
 
@@ -980,6 +986,7 @@ extern "C" talaria_status_t talaria_kv_restore_batch(talaria_ctx *ctx, const tal
                                                      const talaria_kv_xfer_t *xfers, int32_t n_xfers,
                                                      void *stream) {
   TAL_ENTER(ctx);
+  CallTimer timer__(ctx, (cudaStream_t)stream, 2);
   if (n_xfers < 0 || (n_xfers > 0 && !xfers)) return TALARIA_ERR_INVALID_ARG;
   TAL_TRY(batch_dup_check(ctx, kv, xfers, n_xfers));
   return kv_batch(ctx, kv, xfers, n_xfers, (cudaStream_t)stream, false);

@@ -616,7 +616,7 @@ static std::mutex g_static_mu;
 static unsigned long long *g_static_addr[kStaticMaxDevices];   // device address, per device
 
 // The array's name is only a host-side handle here; the address a kernel can use has
-// to be asked for, once per device, with that device current.
+// to be asked for, once per device, with that device current.  Called with g_static_mu held.
 static talaria_status_t static_scratch_address(unsigned long long **out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) {
@@ -624,7 +624,6 @@ static talaria_status_t static_scratch_address(unsigned long long **out) {
     return TALARIA_ERR_CUDA;
   }
   if (dev < 0 || dev >= kStaticMaxDevices) return TALARIA_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lk(g_static_mu);
   if (!g_static_addr[dev]) {
     void *ptr = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
@@ -668,6 +667,10 @@ extern "C" talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const i
   const bool derive = (d_sess_hashes == nullptr);
   const int64_t words = cb + (derive ? sb : 0) + tiles;
   if (words > kStaticWords) return TALARIA_ERR_EXTENT;   // beyond the built-in scratch
+  // One host mutex (it allocates nothing) covers the address lookup and BOTH launches: the chain
+  // kernel is a programmatic dependent of the tile kernel enqueued just before it, so two host
+  // threads must not interleave their launches, not even on one stream.
+  std::lock_guard<std::mutex> lk(g_static_mu);
   unsigned long long *scratch = nullptr;
   TAL_TRY(static_scratch_address(&scratch));
   p.pairs = nullptr;

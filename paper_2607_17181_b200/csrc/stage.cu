@@ -256,14 +256,18 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
     e[m] = StageEntry{nullptr, nullptr, 0, tiles, -1, 0};
     TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
     StageParams p{(const StageEntry *)slot->d, (const int32_t *)(slot->d + ent_bytes), m, tiles, nullptr};
+    if (ctx->timing) cudaEventRecord(ctx->tm[2], stream);
     stage_copy_kernel<<<(unsigned)spans, kStageThreads, 0, stream>>>(p);
     TAL_CUDA(ctx, cudaGetLastError());
+    if (ctx->timing) { cudaEventRecord(ctx->tm[3], stream); ctx->tm_d2d = true; }
     ctx->counters.kernel_launches++;
     TAL_TRY(release_slot(ctx, slot, stream));
   }
   // ---- H2D leg, part 2: enqueued second, so the kernel is already running meanwhile
   if (forked) {
+    if (ctx->timing) cudaEventRecord(ctx->tm[4], ctx->reload_stream);
     for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    if (ctx->timing) { cudaEventRecord(ctx->tm[5], ctx->reload_stream); ctx->tm_h2d = true; }
     TAL_CUDA(ctx, cudaEventRecord(ctx->reload_done, ctx->reload_stream));
     TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->reload_done, 0));
   }
@@ -405,14 +409,18 @@ static talaria_status_t plan_run(talaria_ctx *ctx, talaria_stage_plan *sp, const
   }
   if (sp->tiles > 0 && st.d2d_bytes > 0) {
     StageParams p{(const StageEntry *)sp->d_desc, (const int32_t *)(sp->d_desc + sp->ent_bytes), n, sp->tiles, d_bitmap};
+    if (ctx->timing) cudaEventRecord(ctx->tm[2], stream);
     stage_copy_kernel<<<(unsigned)sp->spans, kStageThreads, 0, stream>>>(p);
     TAL_CUDA(ctx, cudaGetLastError());
+    if (ctx->timing) { cudaEventRecord(ctx->tm[3], stream); ctx->tm_d2d = true; }
     ctx->counters.kernel_launches++;
   }
   // (the device bitmap is rewritten by the next run's upload, which the caller orders after
   // this kernel: runs of one prepared plan share a stream or are chained with events)
   if (!runs.empty()) {
+    if (ctx->timing) cudaEventRecord(ctx->tm[4], ctx->reload_stream);
     for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    if (ctx->timing) { cudaEventRecord(ctx->tm[5], ctx->reload_stream); ctx->tm_h2d = true; }
     TAL_CUDA(ctx, cudaEventRecord(ctx->reload_done, ctx->reload_stream));
     TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->reload_done, 0));
   }
@@ -509,6 +517,7 @@ extern "C" talaria_status_t talaria_stage_plan_run(talaria_ctx *ctx, talaria_sta
   std::lock_guard<std::mutex> lk(ctx->mu);
   tal::DeviceGuard g(ctx->device);
   if (!g.ok) return TALARIA_ERR_CUDA;
+  tal::CallTimer timer__(ctx, (cudaStream_t)stream, 3);
   return tal::plan_run(ctx, prepared, dirty_bitmap, stats, (cudaStream_t)stream);
 }
 
@@ -553,5 +562,6 @@ extern "C" talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t
   std::lock_guard<std::mutex> lk(ctx->mu);
   tal::DeviceGuard g(ctx->device);
   if (!g.ok) return TALARIA_ERR_CUDA;
+  tal::CallTimer timer__(ctx, (cudaStream_t)stream, 3);
   return tal::stage_impl(ctx, plan, n, dirty_bitmap, stats, (cudaStream_t)stream);
 }
