@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the KV-substrate hot path on B200 (one process per GPU).
 
-One step = one pass of the whole path for one Qwen3-235B-shaped session
+The timed step is one pass of the whole path for one Qwen3-235B-shaped session
 (94 layers, 4 KV heads, head_dim 128, bf16, 16-token blocks, 25,000-token prefix):
 
     stream A: KV offload of the session's 1,563 scattered blocks to pinned host
@@ -12,7 +12,13 @@ One step = one pass of the whole path for one Qwen3-235B-shaped session
     KV restore of the matched 1,500 blocks into a different free-block permutation
 
 `value` is host-link payload GB/s (offload + restore bytes) over the whole step.
-Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle instead.
+Prints ONE JSON line on rank 0.  After the timed steps the same run measures the other
+configurations and adds them to that line: "configs2" (105,000-token session, 16- and 32-token
+blocks, restore into isolated blocks, overlapped second offload), "configs3" (session-replay mix
+under a 60 GB pool, whole-session eviction vs background checkpoints), "configs4" (59 GB staged
+switch at 0 / 1 / 36 % dirty chunks, with and without a concurrent restore) and "prefix" (one pair
+at session sizes, batch of 1,024 x 32,768 tokens).  `--workload X` prints one of them alone;
+`--workload session` only the timed step.  `--impl reference` times the CPU oracle instead.
 """
 from __future__ import annotations
 
@@ -139,12 +145,17 @@ def oracle_step_factory(layers: int, stage_fraction: float):
         orc.kv_restore(oshape, planes, bt2, 0, nr, image, strides)
         return (n + nr) * shape.bytes_per_block
 
-    sample = (f"{layers} of 94 layers of the same session (offload {n} + restore 1500 blocks), full "
-              f"27k/25k-token match, first {stage_fraction:.3f} of the staging plan; single thread")
+    sample = (f"{layers} of 94 layers of the same session (offload {n} + restore 1500 blocks) and the same "
+              f"fraction ({stage_fraction:.3f}) of the staging plan, full 27k/25k-token match; single thread")
     return step, sample
 
 
-def time_oracle(steps: int, warmup: int, layers: int = 24, stage_fraction: float = 1 / 16):
+# the CPU arm samples the KV layers and the staging plan with ONE fraction
+ORACLE_LAYERS = 12
+ORACLE_FRACTION = ORACLE_LAYERS / 94
+
+
+def time_oracle(steps: int, warmup: int, layers: int = ORACLE_LAYERS, stage_fraction: float = ORACLE_FRACTION):
     step, sample = oracle_step_factory(layers, stage_fraction)
     for _ in range(warmup):
         step()
@@ -192,10 +203,49 @@ def link_ceiling(torch, dev, nbytes=1 << 30, reps=6):
     return best
 
 
-def run_other_workload(args):
-    """configs[2..4]: measurement lines of their own (the default line is configs[1])."""
-    import torch
+def _release_memory(torch):
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    try:
+        torch._C._host_emptyCache()              # pinned blocks cached by torch
+    except Exception:
+        pass
+
+
+def run_leg(name, torch, dev, ceilings, hbm_peak):
+    """One of the other configurations; returns its dict (or the error that stopped it)."""
     import bench_configs as bc
+    units = {
+        "long": "GB/s restore into isolated blocks (mean over cases)",
+        "stage": "GB/s read+write of the D2D staging kernel, all chunks clean, alone",
+        "replay": "GB/s restore of returning sessions (background-checkpoint mode)",
+        "prefix": "tokens/s, batch of 1,024 pairs x 32,768 tokens, both streams hashed",
+        "sweep": "GB/s best bounce-variant offload of the 25,000-token session",
+    }
+    t0 = time.perf_counter()
+    try:
+        if name == "long":
+            res = bc.run_long(torch, dev, ceilings)
+        elif name == "stage":
+            res = bc.run_stage(torch, dev, ceilings, hbm_peak)
+        elif name == "replay":
+            res = bc.run_replay(torch, dev, ceilings)
+        elif name == "prefix":
+            res = bc.run_prefix(torch, dev, hbm_peak)
+        else:
+            res = bc.run_sweep(torch, dev, ceilings)
+        res["unit"] = units[name]
+    except Exception as e:                        # a leg that cannot run here (memory) must not lose the line
+        res = {"error": f"{type(e).__name__}: {e}"}
+    res["seconds"] = time.perf_counter() - t0
+    _release_memory(torch)
+    return res
+
+
+def run_other_workload(args):
+    """One of configs[2..4] / prefix / sweep as a line of its own."""
+    import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -205,24 +255,11 @@ def run_other_workload(args):
     peaks, kind = measured_peaks()
     sampler = ClockSampler(local)
     sampler.start()
-    if args.workload == "long":
-        res = bc.run_long(torch, dev, ceilings)
-        unit = "GB/s restore into isolated blocks (mean over cases)"
-    elif args.workload == "stage":
-        res = bc.run_stage(torch, dev, ceilings, float(peaks["hbm_gbs"]))
-        unit = "GB/s read+write of the D2D staging kernel, all chunks clean, alone"
-    elif args.workload == "sweep":
-        res = bc.run_sweep(torch, dev, ceilings)
-        unit = "GB/s best bounce-variant offload of the 25,000-token session"
-    elif args.workload == "prefix":
-        res = bc.run_prefix(torch, dev)
-        unit = "tokens/s, batch of 1,024 pairs x 32,768 tokens, both streams hashed"
-    else:
-        res = bc.run_replay(torch, dev, ceilings)
-        unit = "GB/s aggregate offload+restore payload over the drained transfer calls"
+    res = run_leg(args.workload, torch, dev, ceilings, float(peaks["hbm_gbs"]))
     clocks = sampler.stop()
-    line = {"metric": METRIC, "value": res.pop("value"), "unit": unit, "n_gpus": 1, "higher_is_better": True,
-            "dtype": "u8", "data": "synthetic", "vs_baseline": None, "config": {"workload": res.pop("workload")},
+    line = {"metric": METRIC, "value": res.pop("value", None), "unit": res.pop("unit", None), "n_gpus": 1,
+            "higher_is_better": True, "dtype": "u8", "data": "synthetic", "vs_baseline": None,
+            "config": {"workload": res.pop("workload", args.workload)},
             "ceilings": {"h2d_gbs": ceilings["h2d"], "d2h_gbs": ceilings["d2h"], "hbm_gbs": peaks["hbm_gbs"],
                          "hbm_kind": kind, "nominal_pcie5_x16_gbs": PCIE5_X16_GBS}, "clocks": clocks}
     line.update(res)
@@ -322,9 +359,8 @@ def run_gpu(args):
                                   wl.HASH_SEED, h_hashes.numpy().view(np.uint64), h_match, stream=sa)
             reusable = int(h_match[0]["reusable_tokens"])
         else:
-            ctx.prefix_match(1, d_cont, co, d_sess, so, d_stored, 16, wl.HASH_SEED, d_hashes, d_res, stream=sa)
-            with torch.cuda.stream(sa):
-                h_res.copy_(d_res, non_blocking=True)
+            # the result record is written by the kernel straight into pinned host memory
+            ctx.prefix_match(1, d_cont, co, d_sess, so, d_stored, 16, wl.HASH_SEED, d_hashes, h_res, stream=sa)
             ctx.sync(sa)
             reusable = int(h_res[2])
         if record: m["match"][1].record(sa)
@@ -342,6 +378,8 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    step_ms = []
+
     def timed(e2e: bool):
         for _ in range(args.warmup):
             step(e2e, False)
@@ -351,10 +389,14 @@ def run_gpu(args):
         e0, e1 = ev(), ev()
         e0.record()
         nr = 0
+        bounds = [e0]
         for _ in range(args.steps):
             nr = step(e2e, True)
+            bounds.append(ev())
+            bounds[-1].record()
         e1.record()
         barrier()
+        step_ms[:] = [a.elapsed_time(b) for a, b in zip(bounds[:-1], bounds[1:])]
         ms, _ = job_totals(e0.elapsed_time(e1), 0.0, dist if world > 1 else None, dev)
         return ms / args.steps, nr, ctx.get_counters()
 
@@ -362,6 +404,8 @@ def run_gpu(args):
     sampler.start()
     ms_step, nr, counters = timed(False)
     clocks = sampler.stop()
+    step_stats = {"mean": ms_step, "median": statistics.median(step_ms), "min": min(step_ms), "max": max(step_ms),
+                  "note": "per-step times from CUDA events on the default stream between steps (each step ends drained)"}
     phase = {k: statistics.mean(m[k][0].elapsed_time(m[k][1]) for m in marks)
              for k in ("offload", "stage", "match", "restore") if not (k == "stage" and not len(plan_arr))}
     variant_used = int(counters.last_variant)
@@ -398,6 +442,18 @@ def run_gpu(args):
         torch.cuda.synchronize()
         stage_alone_ms = g0.elapsed_time(g1) / 5
 
+    # prefix match of this session on the GPU alone: events around 100 back-to-back calls
+    for _ in range(3):
+        ctx.prefix_match(1, d_cont, co, d_sess, so, d_stored, 16, wl.HASH_SEED, d_hashes, d_res, stream=sa)
+    ctx.sync(sa)
+    g0, g1 = ev(), ev()
+    g0.record(sa)
+    for _ in range(100):
+        ctx.prefix_match(1, d_cont, co, d_sess, so, d_stored, 16, wl.HASH_SEED, d_hashes, d_res, stream=sa)
+    g1.record(sa)
+    ctx.sync(sa)
+    match_gpu_us = g0.elapsed_time(g1) * 10.0
+
     off_bytes, res_bytes = n * shape.bytes_per_block, nr * shape.bytes_per_block
     link_bytes = off_bytes + res_bytes
     value = world * link_bytes / (ms_step * 1e6)
@@ -419,11 +475,22 @@ def run_gpu(args):
             check &= bool(torch.equal(pl[int(bt[i]) * C:(int(bt[i]) + 1) * C].cpu(), chunk))
             if i < nr:
                 check &= bool(torch.equal(pl[int(bt2[i]) * C:(int(bt2[i]) + 1) * C].cpu(), chunk))
-        r = d_res.cpu().numpy()
+        r = h_res.numpy()
         check &= [int(r[0]), int(r[1]), int(r[2]), int(r[3]) & 0xFFFFFFFF] == [SHARED_TOKENS, SHARED_TOKENS // 16, SHARED_TOKENS // 16 * 16, 0]
         if len(plan_arr):
             for off, nb, _ in (plan[0], plan[len(plan) // 2], plan[-1]):
                 check &= bool(torch.equal(slots[off:off + nb], staging[off:off + nb]))
+
+    # ---- the other configurations, in the same run (rank 0 of a 1-GPU run; replicas only time the step)
+    legs = {}
+    if world == 1 and args.workload == "all":
+        peaks0, _ = measured_peaks()
+        ctx.stage_plan_destroy(prepared) if prepared is not None else None
+        ctx.destroy()
+        del planes, staging, slots, image, kv, _keep
+        _release_memory(torch)
+        for key, name in (("prefix", "prefix"), ("configs2", "long"), ("configs4", "stage"), ("configs3", "replay")):
+            legs[key] = run_leg(name, torch, dev, ceilings, float(peaks0["hbm_gbs"]))
 
     if rank != 0:
         if world > 1:
@@ -474,7 +541,7 @@ def run_gpu(args):
                    "pool_blocks": POOL_BLOCKS, "host_layout": "page-first", "stage_chunk_bytes": STAGE_CHUNK,
                    "stage_bytes": stage_bytes, "variant": variant_used, "replicas": world, "scale": args.scale,
                    "l2": "every op streams inputs far larger than the 126 MB L2 (4.8 GB / 59 GB)"},
-        "phases_ms": phase, "self_check": check,
+        "ms_per_step_stats": step_stats, "phases_ms": phase, "self_check": check,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": res_bytes + (CONT_TOKENS + PREFIX_TOKENS) * 4 + (PREFIX_TOKENS // 16) * 8 + (n + nr) * 4,
                 "d2h_bytes_per_step": off_bytes + 32 + (CONT_TOKENS // 16) * 8},
@@ -486,9 +553,12 @@ def run_gpu(args):
                        "frac": 2 * off_bytes / (gather_ms["gather"] * 1e6) / hbm_peak,
                        "algorithmic_bytes": 2 * off_bytes, "timed": "alone, after the timed steps, 5 launches"},
         "cpu_baseline": cpu, "clocks": clocks,
-        "prefix_match": {"us_per_call": phase["match"] * 1e3,
-                         "tokens_per_s": (CONT_TOKENS + PREFIX_TOKENS) / (phase["match"] * 1e-3)},
+        "prefix_match": {"us_per_call_gpu": match_gpu_us,
+                         "tokens_per_s_gpu": (CONT_TOKENS + PREFIX_TOKENS) / (match_gpu_us * 1e-6),
+                         "timed": "CUDA events around 100 back-to-back calls on one stream, stored hashes supplied",
+                         "us_in_step_incl_marshalling_result_copy_and_sync": phase["match"] * 1e3},
     }
+    line.update(legs)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -502,9 +572,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 zero-copy, 2 bounce+DMA, 3 per-run DMA")
     ap.add_argument("--scale", default="full", choices=["full", "small"], help="small = profiling-sized workload")
-    ap.add_argument("--workload", default="session", choices=["session", "long", "stage", "replay", "sweep", "prefix"],
-                    help="session = configs[1] (the benchmark line); long / replay / stage = configs[2] / [3] / [4]; "
-                         "sweep = variant / size table; prefix = match latency and batch throughput")
+    ap.add_argument("--workload", default="all", choices=["all", "session", "long", "stage", "replay", "sweep", "prefix"],
+                    help="all = the timed configs[1] step plus configs[2..4] and the prefix lines as extra keys of the "
+                         "one JSON line; session = the timed step only; long / replay / stage = configs[2] / [3] / [4] "
+                         "alone; sweep = variant / size table; prefix = match latency and batch throughput")
     ap.add_argument("--pack-ctas", type=int, default=0, help="grid of the bounce variant's pack kernels (0 = library default)")
     ap.add_argument("--no-stage", action="store_true")
     ap.add_argument("--no-verify", action="store_true")
@@ -513,7 +584,7 @@ def main():
     apply_scale(args.scale)
     if args.impl == "reference":
         run_reference(args)
-    elif args.workload != "session":
+    elif args.workload not in ("all", "session"):
         run_other_workload(args)
     else:
         run_gpu(args)

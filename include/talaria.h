@@ -80,6 +80,9 @@ typedef struct {
   int32_t pack_ctas;      /* grid size of the bounce variant's pack / unpack kernels; 0 = 64  */
   int64_t host_match_bytes; /* staging (pinned + device, allocated once at create) of            */
                             /* talaria_prefix_match_host; 0 = 16 MiB, at least 1 MiB             */
+  int32_t reload_ctas;      /* grid of the staged switch's host-reload kernel; 0 = built-in.     */
+                            /* Fewer CTAs leave more of the host link to a concurrent restore.   */
+  int32_t reserved;
 } talaria_config_t;
 
 /* Device-side paged KV pool (Sec. 4.3; descriptor fields of App. C "Attention-layout
@@ -199,7 +202,8 @@ talaria_status_t talaria_prefix_match(talaria_ctx *ctx, int32_t n_pairs,
 
 /* Same computation with every array in HOST memory (pageable or pinned).  The inputs are
  * gathered into the context's pinned staging buffer, go to the device in ONE copy, are
- * matched by the same kernels, and hashes and results come back in ONE copy.  Nothing is
+ * matched by the same kernels, and hashes and results are written by those kernels straight
+ * into the pinned staging (no device-to-host copy).  Nothing is
  * allocated or freed: staging was sized at talaria_create (host_match_bytes).  A batch
  * larger than the staging is processed as several sub-batches of whole pairs; a single
  * pair that does not fit is TALARIA_ERR_EXTENT.  Synchronous: returns after the results

@@ -48,7 +48,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 class Config(C.Structure):
     _fields_ = [("bounce_bytes", C.c_int64), ("dma_min_bytes", C.c_int64), ("variant", C.c_int32),
                 ("validate", C.c_int32), ("zc_ctas", C.c_int32), ("pack_ctas", C.c_int32),
-                ("host_match_bytes", C.c_int64)]
+                ("host_match_bytes", C.c_int64), ("reload_ctas", C.c_int32), ("reserved", C.c_int32)]
 
 
 class KvLayout(C.Structure):
@@ -384,10 +384,10 @@ class Talaria:
 
     def __init__(self, device: int = 0, variant: int = VARIANT_AUTO, bounce_bytes: int = 0,
                  dma_min_bytes: int = 0, validate: bool = True, zc_ctas: int = 0, pack_ctas: int = 0,
-                 host_match_bytes: int = 0):
+                 host_match_bytes: int = 0, reload_ctas: int = 0):
         self._h = C.c_void_p()
         cfg = Config(bounce_bytes, dma_min_bytes, variant, 1 if validate else 0, zc_ctas, pack_ctas,
-                     host_match_bytes)
+                     host_match_bytes, reload_ctas, 0)
         rc = lib().talaria_create(C.byref(self._h), device, C.byref(cfg))
         if rc != OK:
             self._h = C.c_void_p()

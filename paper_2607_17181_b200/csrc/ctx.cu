@@ -272,13 +272,16 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
     TAL_CUDA(ctx, cudaMemset(ctx->prefix_counters, 0, 64 * sizeof(unsigned int)));
     TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->prefix_done, cudaEventDisableTiming));
     TAL_TRY(grow(ctx, &ctx->host_tok, (size_t)ctx->cfg.host_match_bytes));
-    TAL_CUDA(ctx, cudaHostAlloc((void **)&ctx->match_pin, ctx->host_tok.cap, cudaHostAllocDefault));
+    TAL_CUDA(ctx, cudaHostAlloc((void **)&ctx->match_pin, ctx->host_tok.cap, cudaHostAllocMapped));
+    TAL_CUDA(ctx, cudaHostGetDevicePointer((void **)&ctx->match_pin_dev, ctx->match_pin, 0));
     // Internal streams run at the highest priority: their kernels are short packing
     // steps that gate copy-engine transfers, so they should not queue behind a long
     // kernel of the caller's (for example a staging copy on another stream).
     int prio_least = 0, prio_greatest = 0;
     TAL_CUDA(ctx, cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
-    TAL_CUDA(ctx, cudaStreamCreateWithPriority(&ctx->reload_stream, cudaStreamNonBlocking, prio_least));
+    // highest priority as well: the reload kernel is a handful of CTAs that must find SM slots while
+    // the D2D gather, launched just before it with a grid far larger than the GPU, is still running
+    TAL_CUDA(ctx, cudaStreamCreateWithPriority(&ctx->reload_stream, cudaStreamNonBlocking, prio_greatest));
     for (cudaEvent_t &e : ctx->tm) TAL_CUDA(ctx, cudaEventCreate(&e));
     TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->reload_fork, cudaEventDisableTiming));
     TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->reload_done, cudaEventDisableTiming));

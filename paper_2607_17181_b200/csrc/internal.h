@@ -70,6 +70,7 @@ struct talaria_ctx {
   cudaStream_t prefix_stream = nullptr;  // stream of that call (same stream: already ordered)
   tal::DevBuf host_tok;               // device side of talaria_prefix_match_host's staging (fixed size)
   char *match_pin = nullptr;          // pinned side, same size and layout
+  char *match_pin_dev = nullptr;      // ... as the device sees it (results are written through this mapping)
   std::vector<std::pair<char *, size_t>> registered;
   tal::RangeCache host_ranges;        // pinned host allocations seen so far
   tal::RangeCache dev_ranges;         // device allocations seen so far

@@ -564,8 +564,7 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
     if (q1 == q0) return TALARIA_ERR_EXTENT;       // one pair alone is larger than the staging
     const int32_t m = q1 - q0;
     const size_t o_cont = 0, o_sess = o_cont + up((size_t)nc * 4), o_sh = o_sess + up((size_t)ns * 4),
-                 o_ch = o_sh + up(h_sess_hashes ? (size_t)sb * 8 : 0), o_res = o_ch + up((size_t)cb * 8),
-                 o_end = o_res + up((size_t)m * sizeof(talaria_match_t));
+                 o_ch = o_sh + up(h_sess_hashes ? (size_t)sb * 8 : 0), o_res = o_ch + up((size_t)cb * 8);
     const int64_t c0 = cont_offsets[q0], s0 = sess_offsets[q0];
     co.resize((size_t)m + 1);
     so.resize((size_t)m + 1);
@@ -581,13 +580,14 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
       TAL_CUDA(ctx, cudaMemcpyAsync(dev, pin, o_ch, cudaMemcpyHostToDevice, stream));
       ctx->counters.memcpy_calls++;
     }
+    // Hashes and results are written by the kernels straight into the pinned staging (through its
+    // device mapping): a few kilobytes of posted writes, and no device-to-host copy that would
+    // queue behind bulk checkpoint traffic on the copy engine.
+    char *const pin_dev = ctx->match_pin_dev;
     TAL_TRY(prefix_launch(ctx, m, (const int32_t *)(dev + o_cont), co.data(), (const int32_t *)(dev + o_sess),
                           so.data(), h_sess_hashes ? (const uint64_t *)(dev + o_sh) : nullptr, B, seed,
-                          (uint64_t *)(dev + o_ch), (talaria_match_t *)(dev + o_res), stream));
-    // hashes and results come back in one copy
-    const size_t out_from = (h_cont_hashes_out && cb) ? o_ch : o_res;
-    TAL_CUDA(ctx, cudaMemcpyAsync(pin + out_from, dev + out_from, o_end - out_from, cudaMemcpyDeviceToHost, stream));
-    ctx->counters.memcpy_calls++;
+                          (h_cont_hashes_out && cb) ? (uint64_t *)(pin_dev + o_ch) : nullptr,
+                          (talaria_match_t *)(pin_dev + o_res), stream));
     TAL_CUDA(ctx, cudaStreamSynchronize(stream));
     if (h_cont_hashes_out && cb) memcpy(h_cont_hashes_out + cb_before, pin + o_ch, (size_t)cb * 8);
     memcpy(h_results + q0, pin + o_res, (size_t)m * sizeof(talaria_match_t));

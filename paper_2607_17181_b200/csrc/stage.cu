@@ -9,9 +9,12 @@
 // on purpose: staging runs next to KV offload / restore on other streams, and
 // short CTAs let the hardware scheduler interleave those kernels instead of
 // making them wait for a resident grid to drain.  The host precomputes the plan
-// entry each span starts in, so no CTA searches.  The H2D leg is issued on an
-// internal stream as copy-engine copies, merged over neighbouring chunks, and
-// overlaps the kernel.
+// entry each span starts in, so no CTA searches.  The H2D leg runs on an internal
+// stream next to the kernel: a handful of host-sourced runs go through the copy
+// engine; many of them (thousands of scattered dirty chunks) are read by a second,
+// small launch of the same kernel straight from the device-mapped pinned host copy,
+// so the host thread is not held for the length of the transfer by thousands of
+// copy calls and a restore issued meanwhile shares the link instead of queueing.
 #include <algorithm>
 #include <cstring>
 
@@ -21,6 +24,7 @@ namespace tal {
 
 struct StageEntry {
   const char *src;  // null: the chunk has no staged copy (always host-sourced)
+  const char *src_host;  // device-visible alias of the pinned authoritative copy, or null
   char *dst;
   int64_t bytes;
   int64_t tile0;    // first tile of this entry
@@ -34,19 +38,63 @@ constexpr int kSpanTiles = 8;                        // tiles per CTA (512 KiB)
 
 struct StageParams {
   const StageEntry *entries;   // DEVICE [n + 1]; entries[n].tile0 = total tiles
-  const int32_t *span_entry;   // DEVICE [grid]: entry that holds the span's first tile
+  const int32_t *span_entry;   // DEVICE [spans]: entry that holds the span's first tile
   int64_t n;
   int64_t tiles;
-  const uint8_t *dirty;        // DEVICE bitmap or null (prepared plans): dirty entries are left to the host leg
+  const uint8_t *dirty;        // DEVICE bitmap or null: which entries are host-sourced this time
+  int32_t host_leg;            // 0: copy the clean staged entries; 1: copy the host-sourced ones from src_host
 };
 
+// An entry comes from the host when it was never staged or its dirty bit is set; each leg
+// leaves the other leg's entries alone.
 __device__ __forceinline__ bool stage_skip(const StageParams &p, const StageEntry &e) {
-  if (!e.src) return true;
-  return p.dirty && e.chunk_id >= 0 && ((p.dirty[e.chunk_id >> 3] >> (e.chunk_id & 7)) & 1);
+  const bool from_host = !e.src || (p.dirty && e.chunk_id >= 0 && ((p.dirty[e.chunk_id >> 3] >> (e.chunk_id & 7)) & 1));
+  return p.host_leg ? !from_host : from_host;
+}
+
+// One tile (at most 64 KiB) by the whole CTA: four 256-bit loads per thread in flight when the
+// addresses allow, 128-bit or byte accesses otherwise.
+__device__ __forceinline__ void copy_tile(const char *src, char *dst, const int64_t len) {
+  const int tid = threadIdx.x;
+  const uintptr_t low = (uintptr_t)src | (uintptr_t)dst;
+  if ((low & 31) == 0 && len == kStageTile) {
+    Vec32 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) v[k] = ld_cs_32(src + ((size_t)tid + k * kStageThreads) * 32);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) st_cs_32(dst + ((size_t)tid + k * kStageThreads) * 32, v[k]);
+  } else if ((low & 15) == 0) {
+    const int4 *s4 = (const int4 *)src;
+    int4 *d4 = (int4 *)dst;
+    if (len == kStageTile) {
+      int4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = __ldcs(s4 + tid + k * kStageThreads);
+#pragma unroll
+      for (int k = 0; k < 8; ++k) __stcs(d4 + tid + k * kStageThreads, v[k]);
+    } else {
+      const int n16 = (int)(len >> 4);
+      for (int k = tid; k < n16; k += kStageThreads) __stcs(d4 + k, __ldcs(s4 + k));
+      for (int k = (n16 << 4) + tid; k < len; k += kStageThreads) dst[k] = src[k];
+    }
+  } else {
+    for (int k = tid; k < len; k += kStageThreads) dst[k] = src[k];
+  }
 }
 
 __global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_constant__ StageParams p) {
-  const int tid = threadIdx.x;
+  if (p.host_leg) {
+    // Host leg: a small grid walks the ENTRIES (most are skipped with one descriptor read) and a CTA
+    // moves a whole host-sourced entry from the mapped pinned copy, tile by tile.
+    for (int64_t e = blockIdx.x; e < p.n; e += gridDim.x) {
+      const StageEntry cur = p.entries[e];
+      if (stage_skip(p, cur)) continue;
+      for (int64_t off = 0; off < cur.bytes; off += kStageTile)
+        copy_tile(cur.src_host + off, cur.dst + off, min((int64_t)kStageTile, cur.bytes - off));
+    }
+    return;
+  }
+  // D2D leg: one CTA per span of tiles
   const int64_t t_begin = (int64_t)blockIdx.x * kSpanTiles;
   const int64_t t_end = min(p.tiles, t_begin + kSpanTiles);
   int64_t e = p.span_entry[blockIdx.x];
@@ -62,36 +110,18 @@ __global__ void __launch_bounds__(kStageThreads) stage_copy_kernel(const __grid_
     }
     if (skip) continue;
     const int64_t off = (t - cur.tile0) * kStageTile;
-    const int64_t len = min((int64_t)kStageTile, cur.bytes - off);
-    const char *src = cur.src + off;
-    char *dst = cur.dst + off;
-    const uintptr_t low = (uintptr_t)src | (uintptr_t)dst;
-    if ((low & 31) == 0 && len == kStageTile) {
-      // full tile, 32-byte aligned: four 256-bit loads per thread in flight
-      Vec32 v[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) v[k] = ld_cs_32(src + ((size_t)tid + k * kStageThreads) * 32);
-#pragma unroll
-      for (int k = 0; k < 4; ++k) st_cs_32(dst + ((size_t)tid + k * kStageThreads) * 32, v[k]);
-    } else if ((low & 15) == 0) {
-      const int4 *s4 = (const int4 *)src;
-      int4 *d4 = (int4 *)dst;
-      if (len == kStageTile) {
-        int4 v[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) v[k] = __ldcs(s4 + tid + k * kStageThreads);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) __stcs(d4 + tid + k * kStageThreads, v[k]);
-      } else {
-        const int n16 = (int)(len >> 4);
-        for (int k = tid; k < n16; k += kStageThreads) __stcs(d4 + k, __ldcs(s4 + k));
-        for (int k = (n16 << 4) + tid; k < len; k += kStageThreads) dst[k] = src[k];
-      }
-    } else {
-      for (int k = tid; k < len; k += kStageThreads) dst[k] = src[k];
-    }
+    copy_tile(cur.src + off, cur.dst + off, min((int64_t)kStageTile, cur.bytes - off));
   }
 }
+
+// Host-sourced runs beyond this count go through the kernel's host leg instead of one
+// copy-engine call each; its grid is small because a few CTAs already saturate the host link.
+constexpr size_t kReloadKernelMinRuns = 32;
+// Measured with 21 GB of scattered 2 MiB reloads (36 % of the chunks dirty): 8 CTAs read 51.4 GB/s
+// from pinned memory, as many as 32 do, and a 25,000-token restore issued meanwhile keeps 35 GB/s
+// of the link (18 GB/s next to a 16- or 32-CTA reload; 39 GB/s next to 4 CTAs, which however
+// no longer hide a 1 % reload under the 18 ms D2D gather).
+static int64_t reload_ctas(const talaria_ctx *ctx) { return ctx->cfg.reload_ctas > 0 ? ctx->cfg.reload_ctas : 8; }
 
 struct Range {
   uintptr_t lo, hi;
@@ -191,6 +221,46 @@ static talaria_status_t check_device_ranges(talaria_ctx *ctx, const talaria_copy
   return TALARIA_OK;
 }
 
+// One leg of a one-shot switch: a compact descriptor (entries, then one int32 per span) is
+// built in a slot, uploaded on `stream` and consumed by one launch on `stream`.
+struct LegItem {
+  const char *src, *src_host;
+  char *dst;
+  int64_t bytes;
+};
+
+static talaria_status_t launch_leg(talaria_ctx *ctx, const std::vector<LegItem> &items, bool host_leg,
+                                   cudaStream_t stream) {
+  int64_t tiles = 0;
+  for (const LegItem &it : items) tiles += (it.bytes + kStageTile - 1) / kStageTile;
+  if (tiles == 0) return TALARIA_OK;
+  const int64_t spans = (tiles + kSpanTiles - 1) / kSpanTiles;
+  if (spans > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
+  const int64_t m = (int64_t)items.size();
+  const size_t ent_bytes = ((size_t)(m + 1) * sizeof(StageEntry) + 15) & ~(size_t)15;
+  const size_t desc_bytes = ent_bytes + (size_t)spans * sizeof(int32_t);
+  DescSlot *slot;
+  TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
+  StageEntry *e = (StageEntry *)slot->h;
+  int32_t *span_entry = (int32_t *)(slot->h + ent_bytes);
+  int64_t t0 = 0, next_span = 0;
+  for (int64_t k = 0; k < m; ++k) {
+    const int64_t nt = (items[(size_t)k].bytes + kStageTile - 1) / kStageTile;
+    e[k] = StageEntry{items[(size_t)k].src, items[(size_t)k].src_host, items[(size_t)k].dst, items[(size_t)k].bytes, t0, -1, 0};
+    // spans whose first tile falls inside this entry
+    while (next_span < spans && next_span * kSpanTiles < t0 + nt) span_entry[next_span++] = (int32_t)k;
+    t0 += nt;
+  }
+  e[m] = StageEntry{nullptr, nullptr, nullptr, 0, tiles, -1, 0};
+  TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
+  StageParams p{(const StageEntry *)slot->d, (const int32_t *)(slot->d + ent_bytes), m, tiles, nullptr, host_leg ? 1 : 0};
+  const unsigned grid = host_leg ? (unsigned)std::min<int64_t>(m, reload_ctas(ctx)) : (unsigned)spans;
+  stage_copy_kernel<<<grid, kStageThreads, 0, stream>>>(p);
+  TAL_CUDA(ctx, cudaGetLastError());
+  ctx->counters.kernel_launches++;
+  return release_slot(ctx, slot, stream);
+}
+
 static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
                                    const uint8_t *dirty, talaria_stage_stats_t *stats, cudaStream_t stream) {
   if (n < 0 || (n > 0 && !plan)) return TALARIA_ERR_INVALID_ARG;
@@ -205,25 +275,25 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
 
   // ---- H2D leg, part 1: merge neighbouring host-sourced chunks and check every host
   // source before anything is enqueued, so a rejected plan leaves no partial copy behind.
-  struct HostRun { const char *h; char *d; int64_t bytes; };
-  std::vector<HostRun> runs;
+  std::vector<LegItem> runs;
   for (int64_t k = 0; k < n;) {
     if (!from_host[(size_t)k] || plan[k].bytes == 0) { ++k; continue; }
-    HostRun r{(const char *)plan[k].src_host, (char *)plan[k].dst_dev, plan[k].bytes};
+    LegItem r{nullptr, (const char *)plan[k].src_host, (char *)plan[k].dst_dev, plan[k].bytes};
     int64_t j = k + 1;
-    while (j < n && from_host[(size_t)j] && (const char *)plan[j].src_host == r.h + r.bytes &&
-           (char *)plan[j].dst_dev == r.d + r.bytes) {
+    while (j < n && from_host[(size_t)j] && (const char *)plan[j].src_host == r.src_host + r.bytes &&
+           (char *)plan[j].dst_dev == r.dst + r.bytes) {
       r.bytes += plan[j].bytes;
       ++j;
     }
     void *alias;
-    TAL_TRY(mapped_range(ctx, r.h, r.bytes, &alias));
+    TAL_TRY(mapped_range(ctx, r.src_host, r.bytes, &alias));
+    r.src = (const char *)alias;               // kept beside the host address: the kernel leg reads through it
     runs.push_back(r);
     k = j;
   }
   TAL_TRY(check_device_ranges(ctx, plan, n, from_host.data()));
   // The internal stream forks from the caller's stream BEFORE the D2D kernel is launched, so
-  // the host-sourced copies depend only on earlier work and run next to the kernel.
+  // the host-sourced leg depends only on earlier work and runs next to the kernel.
   const bool forked = !runs.empty();
   if (forked) {
     TAL_CUDA(ctx, cudaEventRecord(ctx->reload_fork, stream));
@@ -231,42 +301,25 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   }
   // ---- D2D leg ---------------------------------------------------------------
   if (n_clean > 0 && st.d2d_bytes > 0) {
-    // count tiles first so the descriptor (entries, then one int32 per span) can be sized
-    int64_t tiles = 0;
+    std::vector<LegItem> clean;
+    clean.reserve((size_t)n_clean);
     for (int64_t k = 0; k < n; ++k)
-      if (!from_host[(size_t)k]) tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
-    const int64_t spans = (tiles + kSpanTiles - 1) / kSpanTiles;
-    if (spans > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
-    const size_t ent_bytes = ((size_t)(n_clean + 1) * sizeof(StageEntry) + 15) & ~(size_t)15;
-    const size_t desc_bytes = ent_bytes + (size_t)spans * sizeof(int32_t);
-    DescSlot *slot;
-    TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
-    StageEntry *e = (StageEntry *)slot->h;
-    int32_t *span_entry = (int32_t *)(slot->h + ent_bytes);
-    int64_t m = 0, t0 = 0, next_span = 0;
-    for (int64_t k = 0; k < n; ++k) {
-      if (from_host[(size_t)k]) continue;
-      const int64_t nt = (plan[k].bytes + kStageTile - 1) / kStageTile;
-      e[m] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, t0, -1, 0};
-      // spans whose first tile falls inside this entry
-      while (next_span < spans && next_span * kSpanTiles < t0 + nt) span_entry[next_span++] = (int32_t)m;
-      t0 += nt;
-      ++m;
-    }
-    e[m] = StageEntry{nullptr, nullptr, 0, tiles, -1, 0};
-    TAL_TRY(upload_slot(ctx, slot, desc_bytes, stream));
-    StageParams p{(const StageEntry *)slot->d, (const int32_t *)(slot->d + ent_bytes), m, tiles, nullptr};
+      if (!from_host[(size_t)k]) clean.push_back(LegItem{(const char *)plan[k].src_dev, nullptr, (char *)plan[k].dst_dev, plan[k].bytes});
     if (ctx->timing) cudaEventRecord(ctx->tm[2], stream);
-    stage_copy_kernel<<<(unsigned)spans, kStageThreads, 0, stream>>>(p);
-    TAL_CUDA(ctx, cudaGetLastError());
+    TAL_TRY(launch_leg(ctx, clean, false, stream));
     if (ctx->timing) { cudaEventRecord(ctx->tm[3], stream); ctx->tm_d2d = true; }
-    ctx->counters.kernel_launches++;
-    TAL_TRY(release_slot(ctx, slot, stream));
   }
   // ---- H2D leg, part 2: enqueued second, so the kernel is already running meanwhile
   if (forked) {
     if (ctx->timing) cudaEventRecord(ctx->tm[4], ctx->reload_stream);
-    for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    if (runs.size() > kReloadKernelMinRuns) {
+      std::vector<LegItem> items;
+      items.reserve(runs.size());
+      for (const LegItem &r : runs) items.push_back(LegItem{nullptr, r.src, r.dst, r.bytes});
+      TAL_TRY(launch_leg(ctx, items, true, ctx->reload_stream));
+    } else {
+      for (const LegItem &r : runs) TAL_TRY(enqueue_reload(ctx, r.src_host, r.dst, r.bytes));
+    }
     if (ctx->timing) { cudaEventRecord(ctx->tm[5], ctx->reload_stream); ctx->tm_h2d = true; }
     TAL_CUDA(ctx, cudaEventRecord(ctx->reload_done, ctx->reload_stream));
     TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->reload_done, 0));
@@ -284,6 +337,7 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
 struct talaria_stage_plan {
   std::vector<talaria_copy_t> plan;
   std::vector<uint8_t> host_pinned;   // per entry: its host copy was found pinned when the plan was made
+  std::vector<const char *> host_alias;  // ... and its device-visible alias
   char *d_desc = nullptr;        // entries, then one int32 per span
   size_t ent_bytes = 0;
   int64_t tiles = 0, spans = 0, max_chunk = -1;
@@ -321,11 +375,15 @@ static talaria_status_t plan_create(talaria_ctx *ctx, const talaria_copy_t *plan
   talaria_status_t st = [&]() -> talaria_status_t {
     sp->plan.assign(plan, plan + n);
     sp->host_pinned.assign((size_t)n, 0);
+    sp->host_alias.assign((size_t)n, nullptr);
     for (int64_t k = 0; k < n; ++k) {
       sp->tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
       if (plan[k].chunk_id > sp->max_chunk) sp->max_chunk = plan[k].chunk_id;
-      void *alias;
-      if (plan[k].src_host && mapped_range(ctx, plan[k].src_host, plan[k].bytes, &alias) == TALARIA_OK) sp->host_pinned[(size_t)k] = 1;
+      void *alias = nullptr;
+      if (plan[k].src_host && mapped_range(ctx, plan[k].src_host, plan[k].bytes, &alias) == TALARIA_OK) {
+        sp->host_pinned[(size_t)k] = 1;
+        sp->host_alias[(size_t)k] = (const char *)alias;
+      }
     }
     TAL_TRY(check_device_ranges(ctx, plan, n, nullptr));
     sp->spans = (sp->tiles + kSpanTiles - 1) / kSpanTiles;
@@ -338,11 +396,12 @@ static talaria_status_t plan_create(talaria_ctx *ctx, const talaria_copy_t *plan
     int64_t t0 = 0, next_span = 0;
     for (int64_t k = 0; k < n; ++k) {
       const int64_t nt = (plan[k].bytes + kStageTile - 1) / kStageTile;
-      e[k] = StageEntry{(const char *)plan[k].src_dev, (char *)plan[k].dst_dev, plan[k].bytes, t0, plan[k].chunk_id, 0};
+      e[k] = StageEntry{(const char *)plan[k].src_dev, sp->host_alias[(size_t)k], (char *)plan[k].dst_dev, plan[k].bytes, t0,
+                        plan[k].chunk_id, 0};
       while (next_span < sp->spans && next_span * kSpanTiles < t0 + nt) span_entry[next_span++] = (int32_t)k;
       t0 += nt;
     }
-    e[n] = StageEntry{nullptr, nullptr, 0, sp->tiles, -1, 0};
+    e[n] = StageEntry{nullptr, nullptr, nullptr, 0, sp->tiles, -1, 0};
     TAL_CUDA(ctx, cudaMalloc((void **)&sp->d_desc, desc_bytes));
     TAL_CUDA(ctx, cudaMemcpy(sp->d_desc, host.data(), desc_bytes, cudaMemcpyHostToDevice));
     sp->bitmap_bytes = (size_t)((sp->max_chunk + 8) / 8);
@@ -408,7 +467,7 @@ static talaria_status_t plan_run(talaria_ctx *ctx, talaria_stage_plan *sp, const
     TAL_CUDA(ctx, cudaStreamWaitEvent(ctx->reload_stream, ctx->reload_fork, 0));
   }
   if (sp->tiles > 0 && st.d2d_bytes > 0) {
-    StageParams p{(const StageEntry *)sp->d_desc, (const int32_t *)(sp->d_desc + sp->ent_bytes), n, sp->tiles, d_bitmap};
+    StageParams p{(const StageEntry *)sp->d_desc, (const int32_t *)(sp->d_desc + sp->ent_bytes), n, sp->tiles, d_bitmap, 0};
     if (ctx->timing) cudaEventRecord(ctx->tm[2], stream);
     stage_copy_kernel<<<(unsigned)sp->spans, kStageThreads, 0, stream>>>(p);
     TAL_CUDA(ctx, cudaGetLastError());
@@ -419,7 +478,16 @@ static talaria_status_t plan_run(talaria_ctx *ctx, talaria_stage_plan *sp, const
   // this kernel: runs of one prepared plan share a stream or are chained with events)
   if (!runs.empty()) {
     if (ctx->timing) cudaEventRecord(ctx->tm[4], ctx->reload_stream);
-    for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    if (runs.size() > kReloadKernelMinRuns) {
+      // the resident descriptors already name every entry's pinned copy: the same kernel, told to
+      // take the host-sourced entries, on a grid small enough to leave the SMs to everyone else
+      StageParams p{(const StageEntry *)sp->d_desc, (const int32_t *)(sp->d_desc + sp->ent_bytes), n, sp->tiles, d_bitmap, 1};
+      stage_copy_kernel<<<(unsigned)std::min<int64_t>(n, reload_ctas(ctx)), kStageThreads, 0, ctx->reload_stream>>>(p);
+      TAL_CUDA(ctx, cudaGetLastError());
+      ctx->counters.kernel_launches++;
+    } else {
+      for (const HostRun &r : runs) TAL_TRY(enqueue_reload(ctx, r.h, r.d, r.bytes));
+    }
     if (ctx->timing) { cudaEventRecord(ctx->tm[5], ctx->reload_stream); ctx->tm_h2d = true; }
     TAL_CUDA(ctx, cudaEventRecord(ctx->reload_done, ctx->reload_stream));
     TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->reload_done, 0));

@@ -76,6 +76,7 @@ def test_overstated_capacity_of_a_pinned_or_device_image_is_rejected():
         table = np.arange(n, dtype=np.int32)
         before = _launched(ctx)
         assert _status(ctx.kv_offload, pool.kv, table, 0, n, img.ptr, tb.host_layout(strides, HUGE)) == tb.ERR_EXTENT
+        torch.cuda.empty_cache()
         d_img = torch.zeros(n * shape.bytes_per_block, dtype=torch.uint8, device="cuda")
         assert _status(ctx.kv_gather, pool.kv, table, 0, n, d_img, tb.host_layout(strides, HUGE)) == tb.ERR_EXTENT
         assert _status(ctx.kv_scatter, pool.kv, table, 0, n, d_img, tb.host_layout(strides, HUGE)) == tb.ERR_EXTENT
@@ -120,6 +121,7 @@ def test_stage_ranges_that_leave_their_allocation_are_rejected():
         # their tensor; the other end of each copy sits in the middle of a 192 MiB tensor, so the
         # two ranges of an entry can never meet (that would be an overlap error instead).
         nbytes, too_long, mid = 32 << 20, 36 << 20, 64 << 20
+        torch.cuda.empty_cache()          # no cached block may be larger than the tensor it is handed to
         staging = torch.arange(nbytes // 8, dtype=torch.int64, device="cuda").view(torch.uint8)
         slots = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
         big = torch.zeros(192 << 20, dtype=torch.uint8, device="cuda")
