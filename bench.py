@@ -213,7 +213,7 @@ def _release_memory(torch):
         pass
 
 
-def run_leg(name, torch, dev, ceilings, hbm_peak):
+def run_leg(name, torch, dev, ceilings, hbm_peak, small=False):
     """One of the other configurations; returns its dict (or the error that stopped it)."""
     import bench_configs as bc
     units = {
@@ -232,7 +232,7 @@ def run_leg(name, torch, dev, ceilings, hbm_peak):
         elif name == "replay":
             res = bc.run_replay(torch, dev, ceilings)
         elif name == "prefix":
-            res = bc.run_prefix(torch, dev, hbm_peak)
+            res = bc.run_prefix(torch, dev, hbm_peak, small=small)
         else:
             res = bc.run_sweep(torch, dev, ceilings)
         res["unit"] = units[name]
@@ -255,7 +255,7 @@ def run_other_workload(args):
     peaks, kind = measured_peaks()
     sampler = ClockSampler(local)
     sampler.start()
-    res = run_leg(args.workload, torch, dev, ceilings, float(peaks["hbm_gbs"]))
+    res = run_leg(args.workload, torch, dev, ceilings, float(peaks["hbm_gbs"]), small=args.scale == "small")
     clocks = sampler.stop()
     line = {"metric": METRIC, "value": res.pop("value", None), "unit": res.pop("unit", None), "n_gpus": 1,
             "higher_is_better": True, "dtype": "u8", "data": "synthetic", "vs_baseline": None,

@@ -402,13 +402,15 @@ def run_sweep(torch, dev, ceilings) -> Dict:
             "value": max(b["offload_gbs"] for b in bounce)}
 
 
-def run_prefix(torch, dev, hbm_peak=6542.4) -> Dict:
-    """Prefix-match latency for one returning session and throughput for a large batch."""
+def run_prefix(torch, dev, hbm_peak=6542.4, small=False) -> Dict:
+    """Prefix-match latency for one returning session and throughput for a large batch.
+    small: only the batch, cut to 444 pairs (one wave of the one-CTA-per-pair kernel, 155 MB of
+    tokens) and a few launches: the profiling-sized case."""
     ctx = tb.Talaria(dev.index or 0)
     g = wl.rng(2)
     out = {"workload": "prefix match: one pair at session sizes; batch of 1,024 pairs x 32,768 tokens", "single": []}
     st = torch.cuda.Stream(device=dev)
-    for Ts, Tc, shared in ((25_000, 27_000, 24_000), (105_000, 110_000, 100_000)):
+    for Ts, Tc, shared in (() if small else ((25_000, 27_000, 24_000), (105_000, 110_000, 100_000))):
         sess = wl.tokens(g, Ts)
         cont = wl.continuation(g, sess, Tc, shared)
         d_c, d_s = torch.from_numpy(cont).to(dev), torch.from_numpy(sess).to(dev)
@@ -429,7 +431,7 @@ def run_prefix(torch, dev, hbm_peak=6542.4) -> Dict:
                                   "us_per_call_gpu_back_to_back": back * 1e3, "us_call_plus_sync_via_python": lat * 1e6,
                                   "tokens_per_s_gpu": (Tc + Ts) / back * 1e3,
                                   "self_check": [int(r[0]), int(r[1]), int(r[2])] == [shared, shared // 16, shared // 16 * 16]})
-    npairs, T = 1024, 32768
+    npairs, T = (444 if small else 1024), 32768
     big_c = torch.randint(0, wl.VOCAB, (npairs * T,), dtype=torch.int32, device=dev)
     big_s = big_c.clone()
     big_s[T // 2::T] += 1
@@ -442,7 +444,7 @@ def run_prefix(torch, dev, hbm_peak=6542.4) -> Dict:
     r = d_rb.view(npairs, 4).cpu().numpy()
     ok = bool((r[:, 0] == T // 2).all() and (r[:, 1] == T // 2 // 16).all() and (r[:, 2] == T // 2).all())
     out["batch"] = []
-    reps = 20                                     # back to back, so host-side launch work overlaps the GPU
+    reps = 2 if small else 20                     # back to back, so host-side launch work overlaps the GPU
     for stored in (None, d_stb):
         if stored is not None:                    # the registry's stored hashes: the session streams' own
             for q in range(0, npairs, 128):       # (block_hash takes one stream at a time; done in slices of the batch)
@@ -451,7 +453,7 @@ def run_prefix(torch, dev, hbm_peak=6542.4) -> Dict:
             ctx.sync(st)
         call = lambda: [ctx.prefix_match(npairs, big_c, offs, big_s, offs, stored, 16, wl.HASH_SEED, d_hb, d_rb, stream=st)
                         for _ in range(reps)]
-        ms = _timed(torch, st, call, 5) / reps
+        ms = _timed(torch, st, call, 1 if small else 5) / reps
         r = d_rb.view(npairs, 4).cpu().numpy()
         ok &= bool((r[:, 0] == T // 2).all() and (r[:, 1] == T // 2 // 16).all() and (r[:, 3] & 0xFFFFFFFF == 0).all())
         mixes = npairs * T * (2 if stored is None else 1)
