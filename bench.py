@@ -483,7 +483,7 @@ def run_gpu(args):
 
     # ---- the other configurations, in the same run (rank 0 of a 1-GPU run; replicas only time the step)
     legs = {}
-    if world == 1 and args.workload == "all":
+    if world == 1 and args.workload == "all" and args.scale == "full":
         peaks0, _ = measured_peaks()
         ctx.stage_plan_destroy(prepared) if prepared is not None else None
         ctx.destroy()
