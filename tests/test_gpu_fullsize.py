@@ -27,10 +27,11 @@ def _need(host_gb: float, device_gb: float):
     free_dev, _ = torch.cuda.mem_get_info()
     torch.cuda.empty_cache()
     free_dev = max(free_dev, torch.cuda.mem_get_info()[0])
-    if psutil.virtual_memory().available < host_gb * 1.25e9:
-        pytest.skip(f"needs {host_gb:.0f} GB of free host memory for pinned images")
+    avail = psutil.virtual_memory().available
+    if avail < host_gb * 1.25e9:
+        pytest.skip(f"needs {host_gb * 1.25:.0f} GB of free host memory for pinned images, the box has {avail / 1e9:.0f} GB available")
     if free_dev < device_gb * 1.02e9:
-        pytest.skip(f"needs {device_gb:.0f} GB of free device memory")
+        pytest.skip(f"needs {device_gb * 1.02:.0f} GB of free device memory, the GPU has {free_dev / 1e9:.0f} GB free")
 
 
 def _pool(shape, num_blocks, seed):
