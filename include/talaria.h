@@ -378,7 +378,13 @@ talaria_status_t talaria_kv_scatter(talaria_ctx *ctx, const talaria_kv_layout_t 
  * dirty_bitmap are HOST arrays (bitmap may be NULL = all clean; it must cover the
  * largest chunk_id).  src_host must be pinned where it is used.  Destinations must
  * be pairwise disjoint and disjoint from every staged source that is read
- * (OVERLAP).  stats (HOST, nullable) is filled before return. */
+ * (OVERLAP).  stats (HOST, nullable) is filled before return.
+ * The clean entries are one D2D kernel on `stream`.  The host-sourced entries run
+ * beside it on an internal stream that `stream` then waits for: up to 32 merged runs
+ * as copy-engine copies of at most 32 MiB, more than that as a second, small launch
+ * of the same kernel that reads the pinned copies through their device mapping (the
+ * call returns at once instead of feeding thousands of copies to a full queue, and
+ * a restore issued meanwhile keeps a share of the host link). */
 talaria_status_t talaria_stage(talaria_ctx *ctx, const talaria_copy_t *plan, int64_t n,
                                const uint8_t *dirty_bitmap, talaria_stage_stats_t *stats,
                                void *stream);
