@@ -70,6 +70,61 @@ def test_unaligned_entries(ctx, shift_src, shift_dst):
     _run(ctx, sizes, 48 << 10, 0.1, 0.05, 3, align=1, shift_src=shift_src, shift_dst=shift_dst)
 
 
+@pytest.mark.parametrize("prepared", [False, True])
+@pytest.mark.parametrize("shift", [(0, 0), (16, 0), (1, 3)])
+def test_many_scattered_reloads_take_the_kernels_host_leg(ctx, prepared, shift):
+    """More than 32 separate host-sourced runs: the reload is the staging kernel's second leg, reading
+    the device-mapped pinned copies (aligned, 16-byte and byte paths), not one copy-engine call per run."""
+    sizes = [24_001] * 40 + [300_000, 7, 65_536 * 3, 1 << 20] + [4096] * 60
+    plan, total = wl.stage_plan(sizes, 32 << 10, align=1 if shift != (0, 0) else 256)
+    g = wl.rng(602, 7 * shift[0] + shift[1] + (100 if prepared else 0))
+    n = len(plan)
+    weights = g.integers(0, 256, size=total + 64, dtype=np.uint8)
+    dirty = np.zeros(n, bool)
+    dirty[::2] = True                                                  # every other chunk: no two host runs merge
+    missing = (~dirty) & (g.uniform(size=n) < 0.1)
+    staged = weights.copy()
+    for off, nb, cid in plan:
+        if dirty[cid]:
+            staged[off:off + nb] ^= 0xFF
+    host = GuardedPinned(total + 64); host.np[:] = weights
+    staging = GuardedDevice(total + 64, staged, align_off=shift[0])
+    slots = GuardedDevice(total + 64, np.full(total + 64, 0xEE, np.uint8), align_off=shift[1])
+    arr = np.zeros(n, tb.COPY_DTYPE)
+    for k, (off, nb, cid) in enumerate(plan):
+        arr[k] = (0 if missing[cid] else staging.ptr + off, host.ptr + off, slots.ptr + off, nb, cid, 0)
+    bitmap = np.packbits(dirty, bitorder="little")
+    assert int(dirty.sum() + missing.sum()) > 40
+    ctx.sync()
+    ctx.reset_counters()
+    if prepared:
+        h = ctx.stage_plan_create(arr)
+        st = ctx.stage_plan_run(h, bitmap)
+    else:
+        st = ctx.stage(arr, bitmap)
+    ctx.sync()
+    c = ctx.get_counters()
+    assert c.kernel_launches == 2                                      # the D2D leg and the host leg
+    assert c.memcpy_calls <= 2                                         # descriptor / bitmap uploads only, no per-run copies
+    o_slots = np.full(total + 64, 0xEE, np.uint8)
+    entries = [(None if missing[cid] else off, off, off, nb, cid) for off, nb, cid in plan]
+    ost = orc.stage(staged, weights, o_slots, entries, bitmap)
+    assert np.array_equal(slots.read(), o_slots)
+    assert (st.d2d_bytes, st.h2d_bytes, st.dirty_chunks, st.missing_chunks) == \
+        (ost.d2d_bytes, ost.h2d_bytes, ost.dirty_chunks, ost.missing_chunks)
+    assert np.array_equal(staging.read(), staged) and np.array_equal(host.np, weights)
+    assert slots.guards_ok() and staging.guards_ok() and host.guards_ok()
+    if prepared:
+        # the same plan, next switch: everything clean except what was never staged
+        slots.write(np.full(total + 64, 0xEE, np.uint8))
+        st2 = ctx.stage_plan_run(h, None)
+        ctx.sync()
+        o2 = np.full(total + 64, 0xEE, np.uint8)
+        orc.stage(staged, weights, o2, entries, None)
+        assert np.array_equal(slots.read(), o2) and st2.dirty_chunks == 0
+        ctx.stage_plan_destroy(h)
+
+
 def test_empty_plan_and_zero_byte_entries(ctx):
     st = ctx.stage(np.zeros(0, tb.COPY_DTYPE), None)
     assert (st.d2d_bytes, st.h2d_bytes) == (0, 0)
