@@ -205,7 +205,55 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
         del host
     ctx.destroy()
     out["value"] = out["cases"][0]["d2d_gbs_read_write_alone"]
+    del staging, slots, planes, image
+    torch.cuda.empty_cache()
+    try:
+        out["through_layout"] = _stage_through_layout(torch, dev, total, hbm_peak)
+    except Exception as e:
+        out["through_layout"] = {"error": f"{type(e).__name__}: {e}"}
     return out
+
+
+def _stage_through_layout(torch, dev, weight_bytes, hbm_peak, reps=3) -> Dict:
+    """The same clean switch with every address handed out by the stable-address layout (Sec. 4.2 / 4.4):
+    one 150 GB region, model A active (weights low, runtime buffers high, KV planes in the gap, 30 % of
+    the blocks allocated), model B's 58.96 GB pre-staged in the tails of A's 188 KV planes, gathered
+    into B's weights region at the low end."""
+    S = 150 * 10**9 // 4096 * 4096
+    shape = wl.QWEN235
+    W = -(-weight_bytes // 256) * 256
+    models = [(W, 1 << 30, shape.num_layers, shape.num_planes, shape.chunk_bytes)] * 2
+    region = torch.empty(S, dtype=torch.uint8, device=dev)
+    base = region.data_ptr()
+    pad = (-base) % 256
+    bump = tb.Bump(base + pad, S - 256, models)
+    va = bump.activate(0)
+    ids, _ = bump.alloc_blocks(int(va.num_blocks * 0.3))
+    t0 = time.perf_counter()
+    plan, placed = bump.stage_place(1, 2 << 20)
+    place_ms = (time.perf_counter() - t0) * 1e3
+    slack = bump.staging_slack(1, 2 << 20)
+    # the staged bytes: whatever the tails hold, made random on the device
+    kv_off = va.kv_base - base
+    for o in range(kv_off, kv_off + va.kv_bytes, 1 << 30):
+        m = min(1 << 30, kv_off + va.kv_bytes - o) // 8 * 8
+        region[o:o + m].view(torch.int64).random_()
+    ctx = tb.Talaria(dev.index or 0)
+    st = torch.cuda.Stream(device=dev)
+    prepared = ctx.stage_plan_create(plan)
+    ms = _timed(torch, st, lambda: ctx.stage_plan_run(prepared, None, stream=st), reps)
+    ok = placed == plan.size
+    for k in (0, plan.size // 3, plan.size - 1):
+        e = plan[k]
+        a, d, nb = int(e["src_dev"]) - base, int(e["dst_dev"]) - base, int(e["bytes"])
+        ok &= bool(torch.equal(region[a:a + nb], region[d:d + nb]))
+    ctx.stage_plan_destroy(prepared)
+    ctx.destroy()
+    copied = int(plan["bytes"].sum())
+    return {"region_bytes": S, "pool_blocks": int(va.num_blocks), "allocated_blocks": int(ids.size),
+            "chunks": int(plan.size), "chunks_placed": int(placed), "stage_place_host_ms": place_ms,
+            "staging_slack_bytes_after": int(slack), "stage_ms": ms, "d2d_gbs_read_write": 2 * copied / ms / 1e6,
+            "frac_of_hbm_peak": 2 * copied / ms / 1e6 / hbm_peak, "self_check": bool(ok)}
 
 
 class _Arena:
