@@ -385,6 +385,8 @@ static cudaError_t launch_chain(const PrefixParams &p, int n_pairs, cudaStream_t
   return cudaLaunchKernelEx(&cfg, prefix_chain_kernel, p);
 }
 
+constexpr int64_t kPairKernelMaxTokens = 40960;   // longest pair a small batch gives to a single CTA
+
 // Host side: validates offsets, builds the pair table, sizes scratch, launches.
 static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont,
                                       const int64_t *cont_off, const int32_t *d_sess,
@@ -407,8 +409,14 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   int log2B = -1;
   if (B <= 32 && (B & (B - 1)) == 0)
     while ((1 << ++log2B) < B) {}
-  // Batches with at least one pair per SM: one CTA per pair, one launch, no global scratch.
-  if (!inl && n_pairs >= ctx->sm_count && log2B >= 2)
+  // More than a handful of pairs: one CTA per pair, one launch, no global scratch -- when there is
+  // a pair for every SM, or when no pair is so long that its one CTA would outlast the whole batch
+  // spread over the GPU (measured: 9 to 147 pairs of up to 32,768 tokens take 19-25 us this way
+  // against 22-32 us through the tile and chain kernels; 64 pairs of 131,072 tokens 68 against 54 us).
+  int64_t longest = 0;
+  for (int32_t q = 0; q < n_pairs; ++q)
+    longest = std::max(longest, std::max(cont_off[q + 1] - cont_off[q], sess_off[q + 1] - sess_off[q]));
+  if (!inl && log2B >= 2 && (n_pairs >= ctx->sm_count || longest <= kPairKernelMaxTokens))
     return pair_launch(ctx, n_pairs, d_cont, cont_off, d_sess, sess_off, d_sess_hashes, B, log2B, seed,
                        d_cont_hashes, d_results, stream);
   // A handful of pairs run as ONE fused launch (every pair then owns at least one tile, so some

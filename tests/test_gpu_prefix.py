@@ -126,6 +126,22 @@ def test_ragged_batch_with_degenerate_pairs(ctx, B, with_stored):
     _check_batch(ctx, pairs[:5], B, 0, with_stored, pad_front=3)           # token arrays not 16-byte aligned
 
 
+@pytest.mark.parametrize("with_stored", [False, True])
+def test_small_batch_with_a_long_pair_uses_the_tile_and_chain_kernels(ctx, with_stored):
+    # a dozen pairs, one of them longer than a single CTA should take: the two-kernel path
+    g = wl.rng(511)
+    pairs = []
+    for ts, tc, shared in [(50_000, 52_000, 47_001)] + [(int(g.integers(0, 6000)), int(g.integers(0, 6000)), None) for _ in range(11)]:
+        s = wl.tokens(g, ts)
+        pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1)) if shared is None else shared), s))
+    before = ctx.get_counters().kernel_launches
+    _check_batch(ctx, pairs, 16, SEED, with_stored)
+    assert ctx.get_counters().kernel_launches - before == 2
+    before = ctx.get_counters().kernel_launches
+    _check_batch(ctx, pairs[1:], 16, SEED, with_stored, pad_front=(2, 1))      # without the long pair: one CTA per pair
+    assert ctx.get_counters().kernel_launches - before == 1
+
+
 def test_corrupted_stored_hash_is_reported(ctx):
     g = wl.rng(504)
     s = wl.tokens(g, 1000)
