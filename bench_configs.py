@@ -181,9 +181,9 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
             e[2].record(sb)                               # the restore is timed from the moment it is issued
             ctx.kv_restore(kv, table, 0, nblk, image, hl, stream=sb); e[3].record(sb)
             torch.cuda.synchronize()
-            both.append((e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3])))
+            both.append((e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3]), max(e[0].elapsed_time(e[1]), e[0].elapsed_time(e[3]))))
         ctx.stage_plan_destroy(prepared)
-        t_st, t_rs = min(both, key=lambda x: x[1])
+        t_st, t_rs, t_window = min(both, key=lambda x: x[1])
         d2d = total - h2d
         ok = True
         for k in ([0, n // 2, n - 1] + [int(x) for x in idx[:3]]):
@@ -201,7 +201,9 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
             "restore_alone_gbs": image.numel() / t_res_alone / 1e6,
             "restore_with_stage_gbs": image.numel() / t_rs / 1e6,
             "restore_with_stage_frac_of_h2d_ceiling": image.numel() / t_rs / 1e6 / ceilings["h2d"],
-            "link_sum_with_restore_gbs": (h2d / t_st / 1e6 if h2d else 0.0) + image.numel() / t_rs / 1e6})
+            # all host-to-device bytes of the two operations over the window from the first start to the last end
+            "h2d_link_gbs_over_both": (h2d + image.numel()) / t_window / 1e6,
+            "h2d_link_frac_of_ceiling_over_both": (h2d + image.numel()) / t_window / 1e6 / ceilings["h2d"]})
         del host
     ctx.destroy()
     out["value"] = out["cases"][0]["d2d_gbs_read_write_alone"]
