@@ -27,7 +27,8 @@ struct PairDesc {
   int64_t cont_off, sess_off;          // token offsets into the concatenated arrays
   int64_t Tc, Ts;                      // token counts
   int64_t cont_blk_off, sess_blk_off;  // block offsets into hash / digest arrays
-  int64_t tile_off;                    // first tile of this pair
+  int64_t tile_off;                    // first tile of this pair (tiled kernels); the pair's index
+                                       // in the call (one-CTA-per-pair kernel, whose table is sorted)
 };
 
 constexpr int kInlinePairs = 8;    // up to this many pairs travel in the kernel parameters
@@ -36,7 +37,6 @@ constexpr int64_t kFusedMaxTiles = 296;    // 2 CTAs per SM x 148 SMs: about one
 struct PrefixParams {
   const PairDesc *pairs;      // DEVICE [n_pairs + 1] (last entry holds the totals); null when inline
   const int32_t *tile_pair;   // DEVICE [tiles]: pair of each tile; null when inline
-  const int32_t *order;       // DEVICE [n_pairs]: pairs, longest first (one-CTA-per-pair kernel only)
   PairDesc inl[kInlinePairs + 1];
   int32_t n_pairs;
   int32_t B;

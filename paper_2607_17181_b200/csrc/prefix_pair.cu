@@ -17,6 +17,7 @@
 // case in a concatenated batch) are read with aligned loads and re-aligned in registers.
 // The hashing is bound by the integer ALU pipe (three 64-bit xor-shifts per token).
 #include <algorithm>
+#include <vector>
 
 #include "prefix_common.cuh"
 
@@ -197,8 +198,8 @@ __global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kern
   __shared__ uint64_t s_tot[2][kPairWarps];
   __shared__ long long s_red[2][kPairThreads / 32];
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int pair = p.order[blockIdx.x];
-  const PairDesc pd = p.pairs[pair];
+  const PairDesc pd = p.pairs[blockIdx.x];             // sorted longest first; tile_off = the pair's index
+  const int pair = (int)pd.tile_off;
   const int32_t *cont = p.cont + pd.cont_off;
   const int32_t *sess = p.sess + pd.sess_off;
   const int mc = (int)(((uintptr_t)cont >> 2) & 3), ms = (int)(((uintptr_t)sess >> 2) & 3);
@@ -343,7 +344,8 @@ static void launch_pair_kernel(const PrefixParams &p, int log2B, unsigned grid, 
   }
 }
 
-// Pair table and the longest-first order go up in one descriptor slot; one launch.
+// The pair table is written longest pair first (so the last CTAs to start are the short ones),
+// each entry carrying its pair's index in tile_off; one launch.
 // log2B must be 2..5 (block sizes 4, 8, 16, 32).
 talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont, const int64_t *cont_off,
                              const int32_t *d_sess, const int64_t *sess_off, const uint64_t *d_sess_hashes,
@@ -351,7 +353,7 @@ talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d
                              talaria_match_t *d_results, cudaStream_t stream) {
   if (log2B < 2 || log2B > 5) return TALARIA_ERR_INVALID_ARG;
   const size_t pair_bytes = ((size_t)n_pairs * sizeof(PairDesc) + 15) & ~(size_t)15;
-  const size_t desc_bytes = pair_bytes + (size_t)n_pairs * sizeof(int32_t);
+  const size_t desc_bytes = 2 * pair_bytes;          // second half: the table in call order, before sorting
   // offsets are checked before a slot is taken
   for (int32_t q = 0; q < n_pairs; ++q)
     if (cont_off[q + 1] < cont_off[q] || sess_off[q + 1] < sess_off[q] || cont_off[q] < 0 || sess_off[q] < 0)
@@ -361,24 +363,30 @@ talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d
   DescSlot *slot = nullptr;
   TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
   PairDesc *pd = (PairDesc *)slot->h;
-  int32_t *order = (int32_t *)(slot->h + pair_bytes);
+  PairDesc *in_order = (PairDesc *)(slot->h + pair_bytes);
   int64_t cb = 0, sb = 0;
+  bool sorted = true;
   for (int32_t q = 0; q < n_pairs; ++q) {
     const int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
-    pd[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, 0};
+    in_order[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, q};
     cb += Tc / B;
     sb += Ts / B;
-    order[q] = q;
+    if (q && std::max(Tc, Ts) > std::max(in_order[q - 1].Tc, in_order[q - 1].Ts)) sorted = false;
   }
-  // longest pairs first, so the last CTAs to start are the short ones
-  std::stable_sort(order, order + n_pairs, [&](int32_t a, int32_t b) {
-    return std::max(pd[a].Tc, pd[a].Ts) > std::max(pd[b].Tc, pd[b].Ts);
-  });
-  // Each CTA reads its one descriptor straight from the pinned slot (60 bytes over the host
+  if (sorted) {
+    pd = in_order;
+  } else {
+    std::vector<int32_t> order(n_pairs);
+    for (int32_t q = 0; q < n_pairs; ++q) order[q] = q;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+      return std::max(in_order[a].Tc, in_order[a].Ts) > std::max(in_order[b].Tc, in_order[b].Ts);
+    });
+    for (int32_t q = 0; q < n_pairs; ++q) pd[q] = in_order[order[q]];
+  }
+  // Each CTA reads its one descriptor straight from the pinned slot (56 bytes over the host
   // link): no upload stands between this launch and the previous kernel on the stream.
   PrefixParams p{};
-  p.pairs = (const PairDesc *)slot->h;
-  p.order = (const int32_t *)(slot->h + pair_bytes);
+  p.pairs = pd;
   p.n_pairs = n_pairs;
   p.B = B;
   p.log2B = log2B;
