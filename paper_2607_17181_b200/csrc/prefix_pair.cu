@@ -28,8 +28,7 @@ namespace tal {
 // per cent of each other (the integer ALU pipe is the limit, not occupancy or memory latency).
 constexpr int kPairThreads = 256;
 constexpr int kPairCtasPerSm = 3;      // register budget of 80 per thread
-constexpr int kDepthOne = 2;           // quads in flight when one stream is hashed
-constexpr int kDepthBoth = 1;          // ... per stream when both are hashed
+constexpr int kDepth = 2;              // quads in flight per stream
 constexpr int kPairWarps = kPairThreads / 32;
 constexpr int kChunkBlocks = 1024;                         // blocks per chunk
 constexpr int kRounds = kChunkBlocks / kPairThreads;       // blocks per thread per chunk
@@ -79,14 +78,14 @@ __device__ __forceinline__ void note_mismatch(const int4 a, const int4 b, const 
 
 // Rounds [r0, r1) of a chunk in which every token exists wherever it is used and every block is
 // full.  In round r this thread owns block r*256 + tid of the chunk.  MODE 0: hash cont.
-// MODE 1: hash cont, compare with sess.  MODE 2: hash both, compare.  Quads are requested
-// DEPTH quads before they are mixed (a rolling buffer of DEPTH quads per stream).
+// MODE 1: hash cont, compare with sess.  Quads are requested DEPTH quads before they are used
+// (a rolling buffer of DEPTH quads per stream).
 template <int LOG2B, int MODE, bool ALIGNED>
 __device__ __forceinline__ void hash_blocks(const int32_t *cont, const int32_t *sess, const int mc, const int ms,
                                             const int64_t tbase, const int r0, const int r1, uint64_t *dig_c,
-                                            uint64_t *dig_s, long long &first_mis) {
+                                            long long &first_mis) {
   constexpr int Q = (1 << LOG2B) / 4;                    // quads per block
-  constexpr int DEPTH = Q < 4 ? Q : (MODE == 2 ? kDepthBoth : kDepthOne); // quads in flight per stream
+  constexpr int DEPTH = Q < kDepth ? Q : kDepth;         // quads in flight per stream
   constexpr int kRoundTok = kPairThreads << LOG2B;       // tokens between this thread's blocks of two rounds
   if (r0 >= r1) return;
   const int tid = threadIdx.x;
@@ -103,7 +102,7 @@ __device__ __forceinline__ void hash_blocks(const int32_t *cont, const int32_t *
     }
   }
   for (int r = r0; r < r1; ++r) {
-    uint64_t vc = 0, vs = 0;
+    uint64_t vc = 0;
 #pragma unroll
     for (int u = 0; u < Q; ++u) {
       const int slot = u % DEPTH;
@@ -115,36 +114,34 @@ __device__ __forceinline__ void hash_blocks(const int32_t *cont, const int32_t *
       }
       if (MODE != 0) note_mismatch(qa, qb, g_first + (int64_t)r * kRoundTok + 4 * u, first_mis);
       switch (u) {      // the position weights are immediates
-#define TAL_QUAD(U) case U: vc += quad_digest<4 * U>(qa); if (MODE == 2) vs += quad_digest<4 * U>(qb); break;
+#define TAL_QUAD(U) case U: vc += quad_digest<4 * U>(qa); break;
         TAL_QUAD(0) TAL_QUAD(1) TAL_QUAD(2) TAL_QUAD(3) TAL_QUAD(4) TAL_QUAD(5) TAL_QUAD(6) TAL_QUAD(7)
 #undef TAL_QUAD
       }
     }
     dig_c[r * kPairThreads + tid] = vc;
-    if (MODE == 2) dig_s[r * kPairThreads + tid] = vs;
   }
 }
 
 // The same rounds with every token and block checked against the ends of the two streams.
-template <int LOG2B, bool DERIVE>
+template <int LOG2B>
 __device__ __forceinline__ void hash_blocks_checked(const int32_t *cont, const int32_t *sess, const int mc,
                                                     const int ms, const int64_t tbase, const int r0, const int r1,
                                                     const int64_t Tc, const int64_t Ts, const int64_t hash_c_end,
-                                                    const int64_t hash_s_end, const int64_t cmp_end,
-                                                    uint64_t *dig_c, uint64_t *dig_s, long long &first_mis) {
+                                                    const int64_t cmp_end, uint64_t *dig_c, long long &first_mis) {
   constexpr int B = 1 << LOG2B;
   constexpr int kRoundTok = kPairThreads << LOG2B;
   const int tid = threadIdx.x;
   for (int r = r0; r < r1; ++r) {
     const int64_t gb = tbase + (int64_t)r * kRoundTok + ((int64_t)tid << LOG2B);   // first token of the block
-    const bool full_c = gb < hash_c_end, full_s = DERIVE && gb < hash_s_end;       // a block is full or not hashed
-    uint64_t vc = 0, vs = 0;
-    if (full_c || full_s || gb < cmp_end) {
+    const bool full_c = gb < hash_c_end;                                           // a block is full or not hashed
+    uint64_t vc = 0;
+    if (full_c || gb < cmp_end) {
       for (int j0 = 0; j0 < B; j0 += 4) {
         const int64_t g0 = gb + j0;
         int4 a = make_int4(0, 0, 0, 0), b = make_int4(0, 0, 0, 0);
         if (g0 < Tc && (full_c || g0 < cmp_end)) a = load_quad<false>(cont + g0, mc, g0 + 4 - mc < Tc);
-        if (g0 < Ts && (full_s || g0 < cmp_end)) b = load_quad<false>(sess + g0, ms, g0 + 4 - ms < Ts);
+        if (g0 < Ts && g0 < cmp_end) b = load_quad<false>(sess + g0, ms, g0 + 4 - ms < Ts);
         const int ta[4] = {a.x, a.y, a.z, a.w}, tb[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int e = 3; e >= 0; --e)
@@ -153,12 +150,10 @@ __device__ __forceinline__ void hash_blocks_checked(const int32_t *cont, const i
         for (int e = 0; e < 4; ++e) {
           const uint64_t w = kG * (uint64_t)(j0 + e + 1);
           if (full_c) vc += mix64((uint64_t)(uint32_t)ta[e] + w);
-          if (full_s) vs += mix64((uint64_t)(uint32_t)tb[e] + w);
         }
       }
     }
     dig_c[r * kPairThreads + tid] = vc;
-    if (DERIVE) dig_s[r * kPairThreads + tid] = vs;
   }
 }
 
@@ -194,9 +189,11 @@ __global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kern
   constexpr int B = 1 << LOG2B;
   constexpr int kRoundTok = kPairThreads << LOG2B;     // tokens hashed per round by the whole CTA
   constexpr int kChunkShift = 10 + LOG2B;              // tokens per chunk = 1024 * B
-  __shared__ __align__(16) uint64_t s_dig[DERIVE ? 2 : 1][kChunkBlocks];
-  __shared__ uint64_t s_tot[2][kPairWarps];
+  __shared__ __align__(16) uint64_t s_dig[kChunkBlocks];
+  __shared__ uint64_t s_tot[kPairWarps];
   __shared__ long long s_red[2][kPairThreads / 32];
+  __shared__ unsigned long long s_first;     // DERIVE: the first differing token seen by any thread
+  __shared__ uint64_t s_state;               // DERIVE: chain state before the block that holds it
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const PairDesc pd = p.pairs[blockIdx.x];             // sorted longest first; tile_off = the pair's index
   const int pair = (int)pd.tile_off;
@@ -206,8 +203,11 @@ __global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kern
   const bool aligned = (mc | ms) == 0;
   const int64_t Tc = pd.Tc, Ts = pd.Ts, Tmin = Tc < Ts ? Tc : Ts;
   const int64_t nbc = Tc >> LOG2B, nbs = Ts >> LOG2B, lim = nbc < nbs ? nbc : nbs;
-  const int64_t nb_chain = DERIVE ? (nbc > nbs ? nbc : nbs) : nbc;
-  const int64_t hash_c_end = nbc << LOG2B, hash_s_end = DERIVE ? (nbs << LOG2B) : 0;
+  // Only the continuation is hashed.  With stored hashes the chain compares block by block; when
+  // they are to be derived, every block before the first differing token has equal hashes by
+  // construction, and the session is hashed from that block on until the hashes differ.
+  const int64_t hash_c_end = nbc << LOG2B;
+  if (DERIVE && tid == 0) s_first = (unsigned long long)kNoMismatch;
   const uint64_t *hs_in = DERIVE ? nullptr : p.sess_hashes + pd.sess_blk_off;
   uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_blk_off : nullptr;
 
@@ -223,15 +223,15 @@ __global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kern
       if (n & 1) pow_tid *= b;
   }
 
-  uint64_t carry_c = p.seed, carry_s = p.seed;
+  if (DERIVE) __syncthreads();                        // s_first is set before anyone lowers it
+  uint64_t carry_c = p.seed;
   long long first_mis = kNoMismatch, first_bad = lim;
   bool diverged = false;                              // CTA-uniform: a token mismatch has been seen
   for (int64_t ch = 0;; ++ch) {
     const int64_t tbase = ch << kChunkShift;
     // once the streams have diverged, later session tokens matter only if their hashes are derived
     const int64_t cmp_end = diverged ? 0 : Tmin;
-    int64_t need_end = hash_c_end > hash_s_end ? hash_c_end : hash_s_end;
-    need_end = need_end > cmp_end ? need_end : cmp_end;
+    const int64_t need_end = hash_c_end > cmp_end ? hash_c_end : cmp_end;
     if (tbase >= need_end) break;
     // round r covers tokens [tbase + r*kRoundTok, +kRoundTok): rounds_below(t) of them end at or
     // before t, rounds_reaching(t) of them start before t
@@ -240,67 +240,97 @@ __global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kern
     };
     auto rounds_reaching = [&](int64_t t) { return rounds_below(t + kRoundTok - 1); };
     const int r_end = rounds_reaching(need_end);
-    // [0, r_a): both streams fully present (compare, and hash both when deriving) -- no checks;
-    // [r_a, r_b): rounds that straddle the end of a stream -- checked;
+    // [0, r_a): both streams fully present (hash the continuation, compare) -- no checks;
+    // [r_a, r_b): rounds that straddle the end of the compared range -- checked;
     // [r_b, r_c): only the continuation is left and its blocks are full -- no checks;
     // [r_c, r_end): its ragged tail -- checked.
-    const int64_t both_end = DERIVE ? (lim << LOG2B) : (hash_c_end < cmp_end ? hash_c_end : cmp_end);
-    const int64_t sess_end = hash_s_end > cmp_end ? hash_s_end : cmp_end;     // beyond it the session is not read
+    const int64_t both_end = hash_c_end < cmp_end ? hash_c_end : cmp_end;
     const int r_a = rounds_below(both_end);
-    int r_b = rounds_reaching(sess_end);
+    int r_b = rounds_reaching(cmp_end);                 // beyond cmp_end the session is not read
     r_b = r_b < r_a ? r_a : (r_b > r_end ? r_end : r_b);
     int r_c = rounds_below(hash_c_end);
     r_c = r_c < r_b ? r_b : r_c;
-    uint64_t *dc = s_dig[0], *ds = s_dig[DERIVE ? 1 : 0];
-    if (aligned) hash_blocks<LOG2B, DERIVE ? 2 : 1, true>(cont, sess, mc, ms, tbase, 0, r_a, dc, ds, first_mis);
-    else         hash_blocks<LOG2B, DERIVE ? 2 : 1, false>(cont, sess, mc, ms, tbase, 0, r_a, dc, ds, first_mis);
-    hash_blocks_checked<LOG2B, DERIVE>(cont, sess, mc, ms, tbase, r_a, r_b, Tc, Ts, hash_c_end, hash_s_end, cmp_end,
-                                       dc, ds, first_mis);
-    if (mc == 0) hash_blocks<LOG2B, 0, true>(cont, sess, mc, ms, tbase, r_b, r_c, dc, ds, first_mis);
-    else         hash_blocks<LOG2B, 0, false>(cont, sess, mc, ms, tbase, r_b, r_c, dc, ds, first_mis);
-    hash_blocks_checked<LOG2B, DERIVE>(cont, sess, mc, ms, tbase, r_c, r_end, Tc, Ts, hash_c_end, hash_s_end, cmp_end,
-                                       dc, ds, first_mis);
+    uint64_t *dc = s_dig;
+    if (aligned) hash_blocks<LOG2B, 1, true>(cont, sess, mc, ms, tbase, 0, r_a, dc, first_mis);
+    else         hash_blocks<LOG2B, 1, false>(cont, sess, mc, ms, tbase, 0, r_a, dc, first_mis);
+    hash_blocks_checked<LOG2B>(cont, sess, mc, ms, tbase, r_a, r_b, Tc, Ts, hash_c_end, cmp_end, dc, first_mis);
+    if (mc == 0) hash_blocks<LOG2B, 0, true>(cont, sess, mc, ms, tbase, r_b, r_c, dc, first_mis);
+    else         hash_blocks<LOG2B, 0, false>(cont, sess, mc, ms, tbase, r_b, r_c, dc, first_mis);
+    hash_blocks_checked<LOG2B>(cont, sess, mc, ms, tbase, r_c, r_end, Tc, Ts, hash_c_end, cmp_end, dc, first_mis);
+    const bool was_diverged = diverged;
+    if (DERIVE && !was_diverged && first_mis != kNoMismatch) atomicMin(&s_first, (unsigned long long)first_mis);
     diverged = __syncthreads_or(first_mis != kNoMismatch) != 0;
+    // DERIVE: the block that holds the first differing token, if it is one of this chunk's blocks
+    // that both streams have in full (it can only be found in the chunk that holds it)
+    int q_div = -1;                                      // ... and this thread's run holds it at q_div
+    bool resolve = false;
+    if (DERIVE && diverged && !was_diverged) {
+      const int64_t d = (int64_t)(s_first >> LOG2B);
+      resolve = d < lim;
+      const int64_t rel = d - (ch * kChunkBlocks + (int64_t)tid * kRounds);
+      if (resolve && rel >= 0 && rel < kRounds) q_div = (int)rel;
+    }
+    // its tokens are requested now and used after the chain phase
+    uint32_t div_c = 0, div_s = 0;
+    if (DERIVE && resolve && wid == 0 && lane < B) {
+      const int64_t g = (int64_t)((s_first >> LOG2B) << LOG2B) + lane;
+      div_c = (uint32_t)__ldg(cont + g);
+      div_s = (uint32_t)__ldg(sess + g);
+    }
 
     // ---- chain over this chunk's blocks ----------------------------------
     const int64_t k0 = ch * kChunkBlocks + tid * kRounds;
-    if (ch * kChunkBlocks < nb_chain) {
-      uint64_t vc[kRounds], vs[kRounds], hst[kRounds];
+    if (ch * kChunkBlocks < nbc) {
+      uint64_t vc[kRounds], hst[kRounds];
 #pragma unroll
       for (int q = 0; q < kRounds; ++q) {
         vc[q] = dc[tid * kRounds + q];
-        vs[q] = DERIVE ? ds[tid * kRounds + q] : 0ull;
         hst[q] = (!DERIVE && k0 + q < lim) ? __ldg(hs_in + k0 + q) : 0ull;
       }
-      uint64_t xc = 0, xs = 0;
+      uint64_t xc = 0;
 #pragma unroll
-      for (int q = 0; q < kRounds; ++q) {
-        xc = xc * kP + vc[q];
-        if (DERIVE) xs = xs * kP + vs[q];
-      }
-      uint64_t bw_c, bl_c, tot_c, bw_s = 0, bl_s = 0, tot_s = 0;
-      chunk_scan(xc, s_tot[0], bw_c, bl_c, tot_c);
-      uint64_t sc = carry_c * pow_tid + bw_c * pow_lane + bl_c, ss = 0;
-      if (DERIVE) {
-        chunk_scan(xs, s_tot[1], bw_s, bl_s, tot_s);
-        ss = carry_s * pow_tid + bw_s * pow_lane + bl_s;
-      }
+      for (int q = 0; q < kRounds; ++q) xc = xc * kP + vc[q];
+      uint64_t bw_c, bl_c, tot_c;
+      chunk_scan(xc, s_tot, bw_c, bl_c, tot_c);
+      uint64_t sc = carry_c * pow_tid + bw_c * pow_lane + bl_c;
 #pragma unroll
       for (int q = 0; q < kRounds; ++q) {
         const int64_t k = k0 + q;
+        if (DERIVE && q == q_div) s_state = sc;
         sc = sc * kP + vc[q];
-        if (DERIVE) ss = ss * kP + vs[q];
         if (k < nbc) {
           const uint64_t hc = mix64(sc);
           if (hc_out) hc_out[k] = hc;
-          if (k < lim) {
-            const uint64_t hs = DERIVE ? mix64(ss) : hst[q];
-            if (hs != hc && k < first_bad) first_bad = k;
-          }
+          if (!DERIVE && k < lim && hst[q] != hc && k < first_bad) first_bad = k;
         }
       }
       carry_c = carry_c * pow_p(kChunkBlocks) + tot_c;
-      if (DERIVE) carry_s = carry_s * pow_p(kChunkBlocks) + tot_s;
+    }
+    if (DERIVE && resolve) {     // CTA-uniform, at most once per pair
+      __syncthreads();
+      if (wid == 0) {
+        // Both chains enter block d in the same state.  mix64 is a bijection, so two block hashes
+        // are equal exactly when the states are: walk on until the states differ (the first step,
+        // unless two different blocks have equal digests).
+        uint64_t st_c = s_state, st_s = st_c;
+        int64_t k = (int64_t)(s_first >> LOG2B);
+        const uint64_t w = kG * (uint64_t)(lane + 1);
+        for (; k < lim; ++k) {
+          uint64_t dgc = lane < B ? mix64((uint64_t)div_c + w) : 0ull, dgs = lane < B ? mix64((uint64_t)div_s + w) : 0ull;
+          for (int m = 16; m >= 1; m >>= 1) {
+            dgc += shfl_xor_u64(dgc, m);
+            dgs += shfl_xor_u64(dgs, m);
+          }
+          st_c = st_c * kP + dgc;
+          st_s = st_s * kP + dgs;
+          if (st_c != st_s) break;
+          if (k + 1 < lim && lane < B) {
+            div_c = (uint32_t)__ldg(cont + ((k + 1) << LOG2B) + lane);
+            div_s = (uint32_t)__ldg(sess + ((k + 1) << LOG2B) + lane);
+          }
+        }
+        first_bad = k < first_bad ? k : first_bad;
+      }
     }
   }
 
