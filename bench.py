@@ -220,7 +220,7 @@ def run_leg(name, torch, dev, ceilings, hbm_peak, small=False):
         "long": "GB/s restore into isolated blocks (mean over cases)",
         "stage": "GB/s read+write of the D2D staging kernel, all chunks clean, alone",
         "replay": "GB/s restore of returning sessions (background-checkpoint mode)",
-        "prefix": "tokens/s, batch of 1,024 pairs x 32,768 tokens, both streams hashed",
+        "prefix": "tokens/s, batch of 1,024 pairs x 32,768 tokens, session hashes derived",
         "sweep": "GB/s best bounce-variant offload of the 25,000-token session",
     }
     t0 = time.perf_counter()

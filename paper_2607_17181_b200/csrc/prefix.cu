@@ -385,7 +385,14 @@ static cudaError_t launch_chain(const PrefixParams &p, int n_pairs, cudaStream_t
   return cudaLaunchKernelEx(&cfg, prefix_chain_kernel, p);
 }
 
-constexpr int64_t kPairKernelMaxTokens = 40960;   // longest pair a small batch gives to a single CTA
+// Batches with fewer pairs than SMs: the one-CTA-per-pair kernel takes as long as its longest pair
+// (measured 8.5 us + 0.285 us per 1,024 tokens for a CTA that has its SM to itself), the tile and
+// chain kernels as long as the whole batch spread over the GPU (21 us + 3.2 us per million token
+// positions).  Measured at 16 - 147 pairs of 32,768 - 131,072 tokens; the faster one is predicted
+// right or within 3 us everywhere in that range.
+static bool pair_kernel_is_faster(int64_t longest, int64_t positions) {
+  return 8.5 + 0.285 * (double)longest / 1024.0 <= 21.0 + 3.2 * (double)positions / 1e6;
+}
 
 // Host side: validates offsets, builds the pair table, sizes scratch, launches.
 static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont,
@@ -411,12 +418,14 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     while ((1 << ++log2B) < B) {}
   // More than a handful of pairs: one CTA per pair, one launch, no global scratch -- when there is
   // a pair for every SM, or when no pair is so long that its one CTA would outlast the whole batch
-  // spread over the GPU (measured: 9 to 147 pairs of up to 32,768 tokens take 19-25 us this way
-  // against 22-32 us through the tile and chain kernels; 64 pairs of 131,072 tokens 68 against 54 us).
-  int64_t longest = 0;
-  for (int32_t q = 0; q < n_pairs; ++q)
-    longest = std::max(longest, std::max(cont_off[q + 1] - cont_off[q], sess_off[q + 1] - sess_off[q]));
-  if (!inl && log2B >= 2 && (n_pairs >= ctx->sm_count || longest <= kPairKernelMaxTokens))
+  // spread over the GPU.
+  int64_t longest = 0, positions = 0;
+  for (int32_t q = 0; q < n_pairs; ++q) {
+    const int64_t t = std::max(cont_off[q + 1] - cont_off[q], sess_off[q + 1] - sess_off[q]);
+    longest = std::max(longest, t);
+    positions += std::max<int64_t>(t, 0);
+  }
+  if (!inl && log2B >= 2 && (n_pairs >= ctx->sm_count || pair_kernel_is_faster(longest, positions)))
     return pair_launch(ctx, n_pairs, d_cont, cont_off, d_sess, sess_off, d_sess_hashes, B, log2B, seed,
                        d_cont_hashes, d_results, stream);
   // A handful of pairs run as ONE fused launch (every pair then owns at least one tile, so some

@@ -131,7 +131,7 @@ def test_small_batch_with_a_long_pair_uses_the_tile_and_chain_kernels(ctx, with_
     # a dozen pairs, one of them longer than a single CTA should take: the two-kernel path
     g = wl.rng(511)
     pairs = []
-    for ts, tc, shared in [(50_000, 52_000, 47_001)] + [(int(g.integers(0, 6000)), int(g.integers(0, 6000)), None) for _ in range(11)]:
+    for ts, tc, shared in [(118_000, 120_000, 110_001)] + [(int(g.integers(0, 6000)), int(g.integers(0, 6000)), None) for _ in range(11)]:
         s = wl.tokens(g, ts)
         pairs.append((wl.continuation(g, s, tc, int(g.integers(0, min(ts, tc) + 1)) if shared is None else shared), s))
     before = ctx.get_counters().kernel_launches
