@@ -215,6 +215,38 @@ talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
                                            uint64_t seed, uint64_t *h_cont_hashes_out,
                                            talaria_match_t *h_results, void *stream);
 
+/* Match against streams that already live on the device (Sec. 4.3: the instance keeps a
+ * session's state between its calls; App. A: the new prompt is compared with what the session
+ * held).  The caller owns one DEVICE token array and one DEVICE hash array and hands out places
+ * ("slots", element offsets) in them.  For each pair the new prompt comes from HOST memory
+ * (pageable or pinned), is copied to d_tokens[cont_slot ..) through the context's pinned staging,
+ * is matched there against the stored stream d_tokens[sess_slot .. +sess_tokens), and its
+ * floor(cont_tokens / B) block hashes are written to d_hashes[cont_hash_slot ..): prompt and hashes
+ * stay where the session's next call can name them as its stored stream, so a stored stream never
+ * crosses the host link again.  sess_hash_slot names the stored stream's block hashes in d_hashes;
+ * -1 derives them (all pairs of a call that have a stored block must agree on this, else
+ * TALARIA_ERR_INVALID_ARG).  sess_tokens = 0 is a session with nothing stored.
+ * Checked before anything is copied or launched: every range lies inside its array
+ * (TALARIA_ERR_EXTENT; the arrays themselves inside their device allocations); no prompt or hash
+ * destination overlaps another one or a stored range this call reads (TALARIA_ERR_OVERLAP).
+ * A prompt larger than the staging (host_match_bytes) is TALARIA_ERR_EXTENT; a batch larger than
+ * it runs as sub-batches of whole pairs.  Nothing is allocated.  Synchronous: returns after the
+ * records are in h_results. */
+typedef struct {
+  const int32_t *h_cont_tokens;   /* HOST [cont_tokens] */
+  int64_t cont_tokens;
+  int64_t cont_slot;              /* where the prompt is stored in d_tokens */
+  int64_t cont_hash_slot;         /* where its block hashes are stored in d_hashes */
+  int64_t sess_slot, sess_tokens; /* the stored stream in d_tokens */
+  int64_t sess_hash_slot;         /* its block hashes in d_hashes, or -1 */
+} talaria_resident_pair_t;
+talaria_status_t talaria_prefix_match_resident(talaria_ctx *ctx, int32_t n_pairs,
+                                               const talaria_resident_pair_t *pairs /* HOST */,
+                                               int32_t *d_tokens, int64_t tokens_capacity,
+                                               uint64_t *d_hashes, int64_t hashes_capacity,
+                                               int32_t block_tokens, uint64_t seed,
+                                               talaria_match_t *h_results /* HOST */, void *stream);
+
 /* No counterpart in the paper: an allocation-free form of talaria_prefix_match.
  *
  * Who needs it: a serving process that has handed all of HBM to its own memory

@@ -106,6 +106,12 @@ class Timing(C.Structure):
                 ("op", C.c_int32), ("reserved", C.c_int32)]
 
 
+class ResidentPair(C.Structure):
+    _fields_ = [("h_cont_tokens", C.c_void_p), ("cont_tokens", C.c_int64), ("cont_slot", C.c_int64),
+                ("cont_hash_slot", C.c_int64), ("sess_slot", C.c_int64), ("sess_tokens", C.c_int64),
+                ("sess_hash_slot", C.c_int64)]
+
+
 class KvXfer(C.Structure):
     _fields_ = [("block_table", C.c_void_p), ("first_block", C.c_int64), ("n_blocks", C.c_int64),
                 ("host", C.c_void_p), ("hl", HostLayout)]
@@ -120,6 +126,8 @@ _SIGNATURES = {
     "talaria_block_hash": (C.c_int32, [_P, _P, C.c_int64, C.c_int32, C.c_uint64, _P, _P]),
     "talaria_prefix_match": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
     "talaria_prefix_match_host": (C.c_int32, [_P, C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
+    "talaria_prefix_match_resident": (C.c_int32, [_P, C.c_int32, _P, _P, C.c_int64, _P, C.c_int64, C.c_int32,
+                                                  C.c_uint64, _P, _P]),
     "talaria_prefix_match_static": (C.c_int32, [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_uint64, _P, _P, _P]),
     "talaria_prefix_agree": (C.c_int64, [C.c_int32, _P, _P, C.c_int64]),
     "talaria_registry_create": (C.c_int32, [C.POINTER(_P), C.c_int64]),
@@ -438,6 +446,21 @@ class Talaria:
                                                     block_tokens, C.c_uint64(seed), _ptr(h_cont_hashes_out),
                                                     _ptr(h_results), _stream_ptr(stream)),
                     "talaria_prefix_match_host")
+
+    def prefix_match_resident(self, pairs, d_tokens, d_hashes, block_tokens: int, seed: int, h_results, stream=None):
+        """pairs: sequence of (h_cont_tokens, cont_slot, cont_hash_slot, sess_slot, sess_tokens, sess_hash_slot);
+        d_tokens / d_hashes: the caller's device arrays (int32 / 64-bit elements)."""
+        arr = (ResidentPair * max(len(pairs), 1))()
+        keep = []
+        for q, (cont, cont_slot, cont_hash_slot, sess_slot, sess_tokens, sess_hash_slot) in enumerate(pairs):
+            c = _i32(cont)
+            keep.append(c)
+            arr[q] = ResidentPair(_ptr(c), int(c.size), int(cont_slot), int(cont_hash_slot), int(sess_slot),
+                                  int(sess_tokens), int(sess_hash_slot))
+        self._check(lib().talaria_prefix_match_resident(self._h, len(pairs), C.cast(arr, _P), _ptr(d_tokens),
+                                                        int(d_tokens.numel()), _ptr(d_hashes), int(d_hashes.numel()),
+                                                        block_tokens, C.c_uint64(seed), _ptr(h_results),
+                                                        _stream_ptr(stream)), "talaria_prefix_match_resident")
 
     @staticmethod
     def prefix_match_static(n_pairs: int, d_cont_tokens, cont_offsets, d_sess_tokens, sess_offsets,

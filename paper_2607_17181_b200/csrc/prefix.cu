@@ -239,8 +239,8 @@ __device__ __forceinline__ void chain_body(const PrefixParams &p, const int pair
   const int64_t nb = derive_s ? (nbc > nbs ? nbc : nbs) : nbc;  // blocks to chain
   const uint64_t *dc = p.dig_c + pd.cont_blk_off;
   const uint64_t *ds = derive_s ? p.dig_s + pd.sess_blk_off : nullptr;
-  const uint64_t *hs_in = p.sess_hashes ? p.sess_hashes + pd.sess_blk_off : nullptr;
-  uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_blk_off : nullptr;
+  const uint64_t *hs_in = p.sess_hashes ? p.sess_hashes + pd.sess_hash_off : nullptr;
+  uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_hash_off : nullptr;
 
   if (tid == 0) { s_carry[0] = p.seed; s_carry[1] = p.seed; }
   __syncthreads();
@@ -394,40 +394,47 @@ static bool pair_kernel_is_faster(int64_t longest, int64_t positions) {
   return 8.5 + 0.285 * (double)longest / 1024.0 <= 21.0 + 3.2 * (double)positions / 1e6;
 }
 
-// Host side: validates offsets, builds the pair table, sizes scratch, launches.
-static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont,
-                                      const int64_t *cont_off, const int32_t *d_sess,
-                                      const int64_t *sess_off, const uint64_t *d_sess_hashes, int32_t B,
-                                      uint64_t seed, uint64_t *d_cont_hashes, talaria_match_t *d_results,
-                                      cudaStream_t stream) {
+// Host side: validates the pairs, builds the pair table, sizes scratch, launches.
+static talaria_status_t prefix_launch_specs(talaria_ctx *ctx, int32_t n_pairs, const PairSpec *specs,
+                                            const int32_t *d_cont, const int32_t *d_sess,
+                                            const uint64_t *d_sess_hashes, int32_t B, uint64_t seed,
+                                            uint64_t *d_cont_hashes, talaria_match_t *d_results,
+                                            cudaStream_t stream) {
   if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
   if (n_pairs == 0) return TALARIA_OK;
-  if (!cont_off || !sess_off) return TALARIA_ERR_INVALID_ARG;
+  if (!specs) return TALARIA_ERR_INVALID_ARG;
   // few pairs: descriptors ride in the kernel parameters (no upload); otherwise a
   // pinned slot holds the pair table followed by one pair index per tile
   const bool inl = n_pairs <= kInlinePairs;
   PrefixParams p{};
   std::vector<PairDesc> big;
   PairDesc *pd = p.inl;
-  if (!inl) {
-    big.resize((size_t)n_pairs + 1);
-    pd = big.data();
-  }
   int log2B = -1;
   if (B <= 32 && (B & (B - 1)) == 0)
     while ((1 << ++log2B) < B) {}
   // More than a handful of pairs: one CTA per pair, one launch, no global scratch -- when there is
   // a pair for every SM, or when no pair is so long that its one CTA would outlast the whole batch
   // spread over the GPU.
-  int64_t longest = 0, positions = 0;
+  int64_t longest = 0, positions = 0, any_c = 0, any_s = 0;
   for (int32_t q = 0; q < n_pairs; ++q) {
-    const int64_t t = std::max(cont_off[q + 1] - cont_off[q], sess_off[q + 1] - sess_off[q]);
+    const PairSpec &sp = specs[q];
+    if (sp.Tc < 0 || sp.Ts < 0 || sp.cont_off < 0 || sp.sess_off < 0 || sp.cont_hash_off < 0 || sp.sess_hash_off < 0)
+      return TALARIA_ERR_INVALID_ARG;
+    const int64_t t = std::max(sp.Tc, sp.Ts);
     longest = std::max(longest, t);
-    positions += std::max<int64_t>(t, 0);
+    positions += t;
+    any_c |= sp.Tc;
+    any_s |= sp.Ts;
   }
+  if (any_c && !d_cont) return TALARIA_ERR_INVALID_ARG;
+  if (any_s && !d_sess) return TALARIA_ERR_INVALID_ARG;
   if (!inl && log2B >= 2 && (n_pairs >= ctx->sm_count || pair_kernel_is_faster(longest, positions)))
-    return pair_launch(ctx, n_pairs, d_cont, cont_off, d_sess, sess_off, d_sess_hashes, B, log2B, seed,
-                       d_cont_hashes, d_results, stream);
+    return pair_launch(ctx, n_pairs, specs, d_cont, d_sess, d_sess_hashes, B, log2B, seed, d_cont_hashes, d_results,
+                       stream);
+  if (!inl) {
+    big.resize((size_t)n_pairs + 1);
+    pd = big.data();
+  }
   // A handful of pairs run as ONE fused launch (every pair then owns at least one tile, so some
   // CTA always finishes it); batches in between use a tile kernel and a chain kernel.
   bool fused = inl;
@@ -437,9 +444,9 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     cb = sb = tiles = 0;
     tile_tok = fused ? kTileTok : kBatchTileTok;
     for (int32_t q = 0; q < n_pairs; ++q) {
-      int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
-      if (Tc < 0 || Ts < 0 || cont_off[q] < 0 || sess_off[q] < 0) return TALARIA_ERR_INVALID_ARG;
-      pd[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, tiles};
+      const PairSpec &sp = specs[q];
+      const int64_t Tc = sp.Tc, Ts = sp.Ts;
+      pd[q] = PairDesc{sp.cont_off, sp.sess_off, Tc, Ts, cb, sb, tiles, sp.cont_hash_off, sp.sess_hash_off};
       cb += Tc / B;
       sb += Ts / B;
       const int64_t t = (std::max(Tc, Ts) + tile_tok - 1) / tile_tok;
@@ -448,9 +455,7 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
     if (!fused || tiles <= kFusedMaxTiles) break;
     fused = false;                        // too much work for one wave of CTAs: lay out again, unfused
   }
-  pd[n_pairs] = PairDesc{cont_off[n_pairs], sess_off[n_pairs], 0, 0, cb, sb, tiles};
-  if (cont_off[n_pairs] > cont_off[0] && !d_cont) return TALARIA_ERR_INVALID_ARG;
-  if (sess_off[n_pairs] > sess_off[0] && !d_sess) return TALARIA_ERR_INVALID_ARG;
+  pd[n_pairs] = PairDesc{0, 0, 0, 0, cb, sb, tiles, 0, 0};      // the totals
   if (tiles > 0x7fffffffll) return TALARIA_ERR_INVALID_ARG;
 
   // The scratch (digests, tile results, counters) is shared by all calls of this context:
@@ -506,6 +511,35 @@ static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const i
   ctx->prefix_busy = true;
   ctx->prefix_stream = stream;
   return slot ? release_slot(ctx, slot, stream) : TALARIA_OK;
+}
+
+// The same for pairs laid out back to back: pair q spans [off[q], off[q+1]) of its token array and
+// its hashes follow those of the pairs before it.
+static talaria_status_t prefix_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont,
+                                      const int64_t *cont_off, const int32_t *d_sess,
+                                      const int64_t *sess_off, const uint64_t *d_sess_hashes, int32_t B,
+                                      uint64_t seed, uint64_t *d_cont_hashes, talaria_match_t *d_results,
+                                      cudaStream_t stream) {
+  if (n_pairs < 0 || B <= 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_pairs == 0) return TALARIA_OK;
+  if (!cont_off || !sess_off) return TALARIA_ERR_INVALID_ARG;
+  PairSpec few[kInlinePairs];
+  std::vector<PairSpec> many;
+  PairSpec *specs = few;
+  if (n_pairs > kInlinePairs) {
+    many.resize((size_t)n_pairs);
+    specs = many.data();
+  }
+  int64_t cb = 0, sb = 0;
+  for (int32_t q = 0; q < n_pairs; ++q) {
+    const int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
+    if (Tc < 0 || Ts < 0 || cont_off[q] < 0 || sess_off[q] < 0) return TALARIA_ERR_INVALID_ARG;
+    specs[q] = PairSpec{cont_off[q], Tc, sess_off[q], Ts, cb, sb};
+    cb += Tc / B;
+    sb += Ts / B;
+  }
+  return prefix_launch_specs(ctx, n_pairs, specs, d_cont, d_sess, d_sess_hashes, B, seed, d_cont_hashes, d_results,
+                             stream);
 }
 
 }  // namespace tal
@@ -616,6 +650,106 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
 }
 
 
+// Match against streams that live on the device (Sec. 4.3: the instance keeps what it knows of a
+// session; App. A: the new prompt is compared with it).  Only the new prompt crosses the host
+// link, and it is left where the next call will find it as the stored stream.
+extern "C" talaria_status_t talaria_prefix_match_resident(talaria_ctx *ctx, int32_t n_pairs,
+                                                          const talaria_resident_pair_t *pairs, int32_t *d_tokens,
+                                                          int64_t tokens_capacity, uint64_t *d_hashes,
+                                                          int64_t hashes_capacity, int32_t B, uint64_t seed,
+                                                          talaria_match_t *h_results, void *stream_) {
+  TAL_ENTER(ctx);
+  cudaStream_t stream = (cudaStream_t)stream_;
+  if (n_pairs < 0 || B <= 0 || tokens_capacity < 0 || hashes_capacity < 0) return TALARIA_ERR_INVALID_ARG;
+  if (n_pairs == 0) return TALARIA_OK;
+  if (!pairs || !h_results) return TALARIA_ERR_INVALID_ARG;
+  // ranges written (prompts, their hashes) and read (stored streams, stored hashes), as [lo, hi)
+  struct Range { int64_t lo, hi; };
+  std::vector<Range> wt, rt, wh, rh;
+  bool any_stored = false, any_derived = false;
+  for (int32_t q = 0; q < n_pairs; ++q) {
+    const talaria_resident_pair_t &r = pairs[q];
+    if (r.cont_tokens < 0 || r.sess_tokens < 0 || (r.cont_tokens > 0 && !r.h_cont_tokens)) return TALARIA_ERR_INVALID_ARG;
+    const int64_t nbc = r.cont_tokens / B, nbs = r.sess_tokens / B;
+    if (r.cont_slot < 0 || r.cont_slot > tokens_capacity - r.cont_tokens) return TALARIA_ERR_EXTENT;
+    if (r.sess_tokens > 0 && (r.sess_slot < 0 || r.sess_slot > tokens_capacity - r.sess_tokens)) return TALARIA_ERR_EXTENT;
+    if (nbc > 0 && (r.cont_hash_slot < 0 || r.cont_hash_slot > hashes_capacity - nbc)) return TALARIA_ERR_EXTENT;
+    if (nbs > 0) {
+      if (r.sess_hash_slot < 0) {
+        any_derived = true;
+      } else {
+        if (r.sess_hash_slot > hashes_capacity - nbs) return TALARIA_ERR_EXTENT;
+        any_stored = true;
+        rh.push_back(Range{r.sess_hash_slot, r.sess_hash_slot + nbs});
+      }
+    }
+    if (r.cont_tokens > 0) wt.push_back(Range{r.cont_slot, r.cont_slot + r.cont_tokens});
+    if (r.sess_tokens > 0) rt.push_back(Range{r.sess_slot, r.sess_slot + r.sess_tokens});
+    if (nbc > 0) wh.push_back(Range{r.cont_hash_slot, r.cont_hash_slot + nbc});
+  }
+  if (any_stored && any_derived) return TALARIA_ERR_INVALID_ARG;      // one mode per call
+  // a prompt (or its hashes) must not land on another prompt or on anything this call still reads
+  auto clash = [](std::vector<Range> &w, const std::vector<Range> &r) {
+    std::sort(w.begin(), w.end(), [](const Range &a, const Range &b) { return a.lo < b.lo; });
+    for (size_t i = 1; i < w.size(); ++i)
+      if (w[i].lo < w[i - 1].hi) return true;
+    for (const Range &x : r) {
+      auto it = std::upper_bound(w.begin(), w.end(), x.lo, [](int64_t v, const Range &a) { return v < a.hi; });
+      if (it != w.end() && it->lo < x.hi) return true;
+    }
+    return false;
+  };
+  if (clash(wt, rt) || clash(wh, rh)) return TALARIA_ERR_OVERLAP;
+  if ((!wt.empty() || !rt.empty()) && !d_tokens) return TALARIA_ERR_INVALID_ARG;
+  if ((!wh.empty() || !rh.empty()) && !d_hashes) return TALARIA_ERR_INVALID_ARG;
+  if (ctx->cfg.validate) {
+    if (d_tokens && tokens_capacity) TAL_TRY(require_device_range(ctx, d_tokens, tokens_capacity * 4));
+    if (d_hashes && hashes_capacity) TAL_TRY(require_device_range(ctx, d_hashes, hashes_capacity * 8));
+  }
+
+  auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+  const size_t cap = ctx->host_tok.cap;
+  char *const pin = ctx->match_pin, *const pin_dev = ctx->match_pin_dev;
+  std::vector<PairSpec> specs;
+  for (int32_t q0 = 0; q0 < n_pairs;) {
+    // the longest run of whole pairs whose prompts and result records fit the pinned staging
+    int32_t q1 = q0;
+    size_t bytes = 0;
+    while (q1 < n_pairs) {
+      const size_t need = bytes + up((size_t)pairs[q1].cont_tokens * 4) + up((size_t)(q1 + 1 - q0) * sizeof(talaria_match_t));
+      if (need > cap) break;
+      bytes += up((size_t)pairs[q1].cont_tokens * 4);
+      ++q1;
+    }
+    if (q1 == q0) return TALARIA_ERR_EXTENT;       // one prompt alone is larger than the staging
+    const int32_t m = q1 - q0;
+    const size_t o_res = bytes;
+    specs.resize((size_t)m);
+    size_t at = 0;
+    for (int32_t q = q0; q < q1; ++q) {
+      const talaria_resident_pair_t &r = pairs[q];
+      // each prompt starts its way to the device as soon as it is in pinned memory
+      if (r.cont_tokens > 0) {
+        memcpy(pin + at, r.h_cont_tokens, (size_t)r.cont_tokens * 4);
+        TAL_CUDA(ctx, cudaMemcpyAsync(d_tokens + r.cont_slot, pin + at, (size_t)r.cont_tokens * 4, cudaMemcpyHostToDevice,
+                                      stream));
+        ctx->counters.memcpy_calls++;
+        at += up((size_t)r.cont_tokens * 4);
+      }
+      specs[(size_t)(q - q0)] = PairSpec{r.cont_slot, r.cont_tokens, r.sess_tokens > 0 ? r.sess_slot : 0, r.sess_tokens,
+                                         r.cont_tokens / B > 0 ? r.cont_hash_slot : 0,
+                                         (any_stored && r.sess_tokens / B > 0) ? r.sess_hash_slot : 0};
+    }
+    TAL_TRY(prefix_launch_specs(ctx, m, specs.data(), d_tokens, d_tokens, any_stored ? d_hashes : nullptr, B, seed,
+                                d_hashes, (talaria_match_t *)(pin_dev + o_res), stream));
+    TAL_CUDA(ctx, cudaStreamSynchronize(stream));
+    memcpy(h_results + q0, pin + o_res, (size_t)m * sizeof(talaria_match_t));
+    q0 = q1;
+  }
+  return TALARIA_OK;
+}
+
+
 // ---------------------------------------------------------------------------
 // Prefix match without any allocation.
 //
@@ -673,12 +807,12 @@ extern "C" talaria_status_t talaria_prefix_match_static(int32_t n_pairs, const i
   for (int32_t q = 0; q < n_pairs; ++q) {
     const int64_t Tc = cont_offsets[q + 1] - cont_offsets[q], Ts = sess_offsets[q + 1] - sess_offsets[q];
     if (Tc < 0 || Ts < 0 || cont_offsets[q] < 0 || sess_offsets[q] < 0) return TALARIA_ERR_INVALID_ARG;
-    p.inl[q] = PairDesc{cont_offsets[q], sess_offsets[q], Tc, Ts, cb, sb, tiles};
+    p.inl[q] = PairDesc{cont_offsets[q], sess_offsets[q], Tc, Ts, cb, sb, tiles, cb, sb};
     cb += Tc / B;
     sb += Ts / B;
     tiles += (std::max(Tc, Ts) + kTileTok - 1) / kTileTok;
   }
-  p.inl[n_pairs] = PairDesc{cont_offsets[n_pairs], sess_offsets[n_pairs], 0, 0, cb, sb, tiles};
+  p.inl[n_pairs] = PairDesc{0, 0, 0, 0, cb, sb, tiles, 0, 0};
   if (cont_offsets[n_pairs] > cont_offsets[0] && !d_cont_tokens) return TALARIA_ERR_INVALID_ARG;
   if (sess_offsets[n_pairs] > sess_offsets[0] && !d_sess_tokens) return TALARIA_ERR_INVALID_ARG;
   const bool derive = (d_sess_hashes == nullptr);

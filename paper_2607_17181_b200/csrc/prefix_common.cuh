@@ -26,9 +26,17 @@ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
 struct PairDesc {
   int64_t cont_off, sess_off;          // token offsets into the concatenated arrays
   int64_t Tc, Ts;                      // token counts
-  int64_t cont_blk_off, sess_blk_off;  // block offsets into hash / digest arrays
+  int64_t cont_blk_off, sess_blk_off;  // block offsets into the scratch digest arrays (packed pair after pair)
   int64_t tile_off;                    // first tile of this pair (tiled kernels); the pair's index
                                        // in the call (one-CTA-per-pair kernel, whose table is sorted)
+  int64_t cont_hash_off, sess_hash_off;  // where the pair's block hashes sit in the callers' hash arrays
+};
+
+// One pair as the host entry points describe it: where its two streams and their block hashes
+// sit in the token and hash arrays (element offsets).
+struct PairSpec {
+  int64_t cont_off, Tc, sess_off, Ts;
+  int64_t cont_hash_off, sess_hash_off;
 };
 
 constexpr int kInlinePairs = 8;    // up to this many pairs travel in the kernel parameters
@@ -62,9 +70,9 @@ __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int d) {
 
 
 // One CTA per pair, for batches with at least one pair per SM (prefix_pair.cu).
-talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont, const int64_t *cont_off,
-                             const int32_t *d_sess, const int64_t *sess_off, const uint64_t *d_sess_hashes,
-                             int32_t B, int log2B, uint64_t seed, uint64_t *d_cont_hashes,
-                             talaria_match_t *d_results, cudaStream_t stream);
+talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const PairSpec *specs, const int32_t *d_cont,
+                             const int32_t *d_sess, const uint64_t *d_sess_hashes, int32_t B, int log2B,
+                             uint64_t seed, uint64_t *d_cont_hashes, talaria_match_t *d_results,
+                             cudaStream_t stream);
 
 }  // namespace tal

@@ -208,8 +208,8 @@ __global__ void __launch_bounds__(kPairThreads, kPairCtasPerSm) prefix_pair_kern
   // construction, and the session is hashed from that block on until the hashes differ.
   const int64_t hash_c_end = nbc << LOG2B;
   if (DERIVE && tid == 0) s_first = (unsigned long long)kNoMismatch;
-  const uint64_t *hs_in = DERIVE ? nullptr : p.sess_hashes + pd.sess_blk_off;
-  uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_blk_off : nullptr;
+  const uint64_t *hs_in = DERIVE ? nullptr : p.sess_hashes + pd.sess_hash_off;
+  uint64_t *hc_out = p.cont_hashes_out ? p.cont_hashes_out + pd.cont_hash_off : nullptr;
 
   // P^(kRounds lane) and P^(kRounds tid): where this thread's run starts inside its warp and inside the chunk
   uint64_t pow_lane = 1, pow_tid = 1;
@@ -377,31 +377,22 @@ static void launch_pair_kernel(const PrefixParams &p, int log2B, unsigned grid, 
 // The pair table is written longest pair first (so the last CTAs to start are the short ones),
 // each entry carrying its pair's index in tile_off; one launch.
 // log2B must be 2..5 (block sizes 4, 8, 16, 32).
-talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const int32_t *d_cont, const int64_t *cont_off,
-                             const int32_t *d_sess, const int64_t *sess_off, const uint64_t *d_sess_hashes,
-                             int32_t B, int log2B, uint64_t seed, uint64_t *d_cont_hashes,
-                             talaria_match_t *d_results, cudaStream_t stream) {
+talaria_status_t pair_launch(talaria_ctx *ctx, int32_t n_pairs, const PairSpec *specs, const int32_t *d_cont,
+                             const int32_t *d_sess, const uint64_t *d_sess_hashes, int32_t B, int log2B,
+                             uint64_t seed, uint64_t *d_cont_hashes, talaria_match_t *d_results,
+                             cudaStream_t stream) {
   if (log2B < 2 || log2B > 5) return TALARIA_ERR_INVALID_ARG;
   const size_t pair_bytes = ((size_t)n_pairs * sizeof(PairDesc) + 15) & ~(size_t)15;
   const size_t desc_bytes = 2 * pair_bytes;          // second half: the table in call order, before sorting
-  // offsets are checked before a slot is taken
-  for (int32_t q = 0; q < n_pairs; ++q)
-    if (cont_off[q + 1] < cont_off[q] || sess_off[q + 1] < sess_off[q] || cont_off[q] < 0 || sess_off[q] < 0)
-      return TALARIA_ERR_INVALID_ARG;
-  if (cont_off[n_pairs] > cont_off[0] && !d_cont) return TALARIA_ERR_INVALID_ARG;
-  if (sess_off[n_pairs] > sess_off[0] && !d_sess) return TALARIA_ERR_INVALID_ARG;
   DescSlot *slot = nullptr;
   TAL_TRY(acquire_slot(ctx, desc_bytes, &slot));
   PairDesc *pd = (PairDesc *)slot->h;
   PairDesc *in_order = (PairDesc *)(slot->h + pair_bytes);
-  int64_t cb = 0, sb = 0;
   bool sorted = true;
   for (int32_t q = 0; q < n_pairs; ++q) {
-    const int64_t Tc = cont_off[q + 1] - cont_off[q], Ts = sess_off[q + 1] - sess_off[q];
-    in_order[q] = PairDesc{cont_off[q], sess_off[q], Tc, Ts, cb, sb, q};
-    cb += Tc / B;
-    sb += Ts / B;
-    if (q && std::max(Tc, Ts) > std::max(in_order[q - 1].Tc, in_order[q - 1].Ts)) sorted = false;
+    const PairSpec &sp = specs[q];
+    in_order[q] = PairDesc{sp.cont_off, sp.sess_off, sp.Tc, sp.Ts, 0, 0, q, sp.cont_hash_off, sp.sess_hash_off};
+    if (q && std::max(sp.Tc, sp.Ts) > std::max(in_order[q - 1].Tc, in_order[q - 1].Ts)) sorted = false;
   }
   if (sorted) {
     pd = in_order;
