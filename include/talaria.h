@@ -136,7 +136,8 @@ typedef struct {
 
 /* App. D "Path classification" also records the D2D and H2D gather times of a switch, and the
  * router charges a measured restore cost (Sec. 3.3): optional per-call timing from CUDA events
- * on the streams the work runs on.  op: 1 offload, 2 restore, 3 stage; the leg fields that do
+ * on the streams the work runs on.  op: 1 offload, 2 restore, 3 stage, 4 prefix match from host
+ * memory (the _host and _resident forms: first copy to last kernel); the leg fields that do
  * not apply are 0.  For a stage, d2d_ms is the gather kernel and h2d_ms the host reloads, which
  * overlap, so total_ms is less than their sum. */
 typedef struct {

@@ -627,6 +627,11 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
     if (nc) memcpy(pin + o_cont, h_cont + c0, (size_t)nc * 4);
     if (ns) memcpy(pin + o_sess, h_sess + s0, (size_t)ns * 4);
     if (h_sess_hashes && sb) memcpy(pin + o_sh, h_sess_hashes + sb_before, (size_t)sb * 8);
+    if (ctx->timing && q0 == 0) {      // op 4: from the first copy to the last kernel, host-side packing excluded
+      ctx->tm_op = 4;
+      ctx->tm_d2d = ctx->tm_h2d = false;
+      TAL_CUDA(ctx, cudaEventRecord(ctx->tm[0], stream));
+    }
     if (o_ch) {
       TAL_CUDA(ctx, cudaMemcpyAsync(dev, pin, o_ch, cudaMemcpyHostToDevice, stream));
       ctx->counters.memcpy_calls++;
@@ -639,6 +644,7 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
                           so.data(), h_sess_hashes ? (const uint64_t *)(dev + o_sh) : nullptr, B, seed,
                           (h_cont_hashes_out && cb) ? (uint64_t *)(pin_dev + o_ch) : nullptr,
                           (talaria_match_t *)(pin_dev + o_res), stream));
+    if (ctx->timing) TAL_CUDA(ctx, cudaEventRecord(ctx->tm[1], stream));
     TAL_CUDA(ctx, cudaStreamSynchronize(stream));
     if (h_cont_hashes_out && cb) memcpy(h_cont_hashes_out + cb_before, pin + o_ch, (size_t)cb * 8);
     memcpy(h_results + q0, pin + o_res, (size_t)m * sizeof(talaria_match_t));
@@ -725,23 +731,41 @@ extern "C" talaria_status_t talaria_prefix_match_resident(talaria_ctx *ctx, int3
     const int32_t m = q1 - q0;
     const size_t o_res = bytes;
     specs.resize((size_t)m);
+    // The prompts are packed in the pinned staging, cross the host link in ONE copy (a copy per
+    // prompt pays the link's latency once each, and several times over while checkpoints keep the
+    // other direction busy), and are spread to their places by device-to-device copies.
     size_t at = 0;
     for (int32_t q = q0; q < q1; ++q) {
       const talaria_resident_pair_t &r = pairs[q];
-      // each prompt starts its way to the device as soon as it is in pinned memory
       if (r.cont_tokens > 0) {
         memcpy(pin + at, r.h_cont_tokens, (size_t)r.cont_tokens * 4);
-        TAL_CUDA(ctx, cudaMemcpyAsync(d_tokens + r.cont_slot, pin + at, (size_t)r.cont_tokens * 4, cudaMemcpyHostToDevice,
-                                      stream));
-        ctx->counters.memcpy_calls++;
         at += up((size_t)r.cont_tokens * 4);
       }
       specs[(size_t)(q - q0)] = PairSpec{r.cont_slot, r.cont_tokens, r.sess_tokens > 0 ? r.sess_slot : 0, r.sess_tokens,
                                          r.cont_tokens / B > 0 ? r.cont_hash_slot : 0,
                                          (any_stored && r.sess_tokens / B > 0) ? r.sess_hash_slot : 0};
     }
+    if (ctx->timing && q0 == 0) {      // op 4: from the first copy to the last kernel, host-side packing excluded
+      ctx->tm_op = 4;
+      ctx->tm_d2d = ctx->tm_h2d = false;
+      TAL_CUDA(ctx, cudaEventRecord(ctx->tm[0], stream));
+    }
+    if (at) {
+      TAL_CUDA(ctx, cudaMemcpyAsync(ctx->host_tok.p, pin, at, cudaMemcpyHostToDevice, stream));
+      ctx->counters.memcpy_calls++;
+      at = 0;
+      for (int32_t q = q0; q < q1; ++q) {
+        const talaria_resident_pair_t &r = pairs[q];
+        if (r.cont_tokens == 0) continue;
+        TAL_CUDA(ctx, cudaMemcpyAsync(d_tokens + r.cont_slot, ctx->host_tok.p + at, (size_t)r.cont_tokens * 4,
+                                      cudaMemcpyDeviceToDevice, stream));
+        ctx->counters.memcpy_calls++;
+        at += up((size_t)r.cont_tokens * 4);
+      }
+    }
     TAL_TRY(prefix_launch_specs(ctx, m, specs.data(), d_tokens, d_tokens, any_stored ? d_hashes : nullptr, B, seed,
                                 d_hashes, (talaria_match_t *)(pin_dev + o_res), stream));
+    if (ctx->timing) TAL_CUDA(ctx, cudaEventRecord(ctx->tm[1], stream));
     TAL_CUDA(ctx, cudaStreamSynchronize(stream));
     memcpy(h_results + q0, pin + o_res, (size_t)m * sizeof(talaria_match_t));
     q0 = q1;

@@ -100,13 +100,16 @@ class ReplayDriver:
                  seed: int, content: Callable[[int, int, int], np.ndarray], alloc_pinned: Callable[[int], object],
                  to_device: Callable[[np.ndarray], object], order: str = "PF", log: Optional[list] = None,
                  free_pinned: Optional[Callable[[object], None]] = None, checkpoint: str = "incremental",
-                 max_extent_blocks: int = 512):
+                 max_extent_blocks: int = 512, resident: Optional[Tuple[int, int]] = None):
         """content(session, call_index, nbytes) -> uint8 array: the synthetic KV of a call's new blocks.
         alloc_pinned(nbytes) -> pinned host tensor; free_pinned(tensor) gives it back (optional);
         to_device(array) -> device tensor (memory plumbing).
         checkpoint: "incremental" (after every call, asynchronously) or "eviction" (whole session when evicted).
         max_extent_blocks: a checkpoint is cut into host images of at most this many blocks, so the
-        pinned allocator is never asked for one multi-gigabyte piece."""
+        pinned allocator is never asked for one multi-gigabyte piece.
+        resident: (sessions, longest prompt) -- keep every session's stream and block hashes on the device
+        (two places per session, used in turn) and match with `talaria_prefix_match_resident`: only the new
+        prompt crosses the host link.  None: every stream goes up from host memory with each match."""
         import torch
         assert checkpoint in ("incremental", "eviction")
         self.ctx, self.shape, self.kv = ctx, shape, kv
@@ -124,6 +127,13 @@ class ReplayDriver:
         self.log = log if log is not None else []
         self._torch = torch
         self.ckpt_stream = torch.cuda.Stream()
+        self.resident = resident
+        if resident is not None:
+            n, longest = resident
+            self.tok_stride, self.hash_stride = longest, longest // shape.block_tokens + 1
+            self.d_tokens = torch.zeros(2 * n * self.tok_stride, dtype=torch.int32, device="cuda")
+            self.d_hashes = torch.zeros(2 * n * self.hash_stride, dtype=torch.int64, device="cuda")
+            self.place: Dict[int, List[int]] = {}            # session -> [index in the arrays, side holding its stream]
 
     # ------------------------------------------------------------ allocation
     def _alloc(self, n: int) -> np.ndarray:
@@ -272,19 +282,37 @@ class ReplayDriver:
             self.sessions.setdefault(sid, SessionState(sid))
         # ---- one batched match for the whole group -------------------------
         conts = [t for _, _, t in calls]
-        sesss = [self.sessions[sid].tokens for sid, _, _ in calls]
-        co = np.cumsum([0] + [c.size for c in conts]).astype(np.int64)
-        so = np.cumsum([0] + [s.size for s in sesss]).astype(np.int64)
-        cont_all = np.concatenate(conts) if co[-1] else np.zeros(1, np.int32)
-        sess_all = np.concatenate(sesss) if so[-1] else np.zeros(1, np.int32)
-        stored = np.concatenate([self.sessions[sid].hashes[: s.size // B] for (sid, _, _), s in zip(calls, sesss)])
-        stored = stored if stored.size else np.zeros(1, np.uint64)
-        out_h = np.zeros(max(int(sum(c.size // B for c in conts)), 1), np.uint64)
         res = np.zeros(len(calls), tb.MATCH_DTYPE)
-        t0 = time.perf_counter()
-        self.ctx.prefix_match_host(len(calls), cont_all, co, sess_all, so, stored, B, self.seed, out_h, res)
-        self.stats.match_s += time.perf_counter() - t0
-        self.stats.match_times.append(time.perf_counter() - t0)
+        if self.resident is not None:
+            pairs, outs = [], []
+            for sid, _, toks in calls:
+                pl = self.place.setdefault(sid, [len(self.place), 0])
+                assert pl[0] < self.resident[0] and toks.size <= self.tok_stride
+                here, there = 2 * pl[0] + pl[1], 2 * pl[0] + (pl[1] ^ 1)
+                pairs.append((toks, there * self.tok_stride, there * self.hash_stride, here * self.tok_stride,
+                              self.sessions[sid].tokens.size, here * self.hash_stride))
+                outs.append((there * self.hash_stride, toks.size // B))
+                pl[1] ^= 1                                    # the prompt becomes the stored stream
+            t0 = time.perf_counter()
+            self.ctx.prefix_match_resident(pairs, self.d_tokens, self.d_hashes, B, self.seed, res)
+            dt = time.perf_counter() - t0
+            got = [self.d_hashes[o:o + n].cpu().numpy().view(np.uint64) for o, n in outs]      # host copies, for the log
+            out_h = np.concatenate(got) if got else np.zeros(0, np.uint64)
+            out_h = out_h if out_h.size else np.zeros(1, np.uint64)
+        else:
+            sesss = [self.sessions[sid].tokens for sid, _, _ in calls]
+            co = np.cumsum([0] + [c.size for c in conts]).astype(np.int64)
+            so = np.cumsum([0] + [s.size for s in sesss]).astype(np.int64)
+            cont_all = np.concatenate(conts) if co[-1] else np.zeros(1, np.int32)
+            sess_all = np.concatenate(sesss) if so[-1] else np.zeros(1, np.int32)
+            stored = np.concatenate([self.sessions[sid].hashes[: s.size // B] for (sid, _, _), s in zip(calls, sesss)])
+            stored = stored if stored.size else np.zeros(1, np.uint64)
+            out_h = np.zeros(max(int(sum(c.size // B for c in conts)), 1), np.uint64)
+            t0 = time.perf_counter()
+            self.ctx.prefix_match_host(len(calls), cont_all, co, sess_all, so, stored, B, self.seed, out_h, res)
+            dt = time.perf_counter() - t0
+        self.stats.match_s += dt
+        self.stats.match_times.append(dt)
         self.stats.match_calls += 1
         self.log.append(("match", [(sid, k) for sid, k, _ in calls], res.copy(), out_h.copy()))
         # ---- residency decisions, allocation ----------------------------------

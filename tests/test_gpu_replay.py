@@ -36,10 +36,11 @@ def _groups(schedule, size):
     return out
 
 
-@pytest.mark.parametrize("order,host_budget_frac,checkpoint", [("PF", 0.35, "eviction"), ("LF", 10.0, "eviction"),
-                                                               ("PF", 10.0, "incremental"), ("LF", 10.0, "incremental"),
-                                                               ("PF", 0.9, "incremental")])
-def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac, checkpoint):
+@pytest.mark.parametrize("order,host_budget_frac,checkpoint,resident",
+                         [("PF", 0.35, "eviction", False), ("LF", 10.0, "eviction", False),
+                          ("PF", 10.0, "incremental", False), ("LF", 10.0, "incremental", True),
+                          ("PF", 0.9, "incremental", True)])
+def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac, checkpoint, resident):
     shape = wl.KvShape(2, 2, 16, 64)
     full = wl.QWEN235
     pool_blocks = int(60e9) // full.bytes_per_block                       # 19,479 blocks, as at the full shape
@@ -56,7 +57,8 @@ def test_session_replay_mix_matches_oracle_mirror(order, host_budget_frac, check
     log = []
     drv = ReplayDriver(ctx, shape, kv, pool_blocks, int(total_kv * host_budget_frac), wl.HASH_SEED, _content,
                        lambda n: torch.empty(n, dtype=torch.uint8, pin_memory=True),
-                       lambda a: torch.from_numpy(a).cuda(), order=order, log=log, checkpoint=checkpoint)
+                       lambda a: torch.from_numpy(a).cuda(), order=order, log=log, checkpoint=checkpoint,
+                       resident=(30, 131_072) if resident else None)
     streams, tg = {}, wl.rng(4, 2)
     try:
         for gi, group in enumerate(_groups(schedule, 4)):

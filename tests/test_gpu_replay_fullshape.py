@@ -85,7 +85,7 @@ def test_session_replay_at_the_full_kv_shape():
     ctx = tb.Talaria(0)
     log = []
     drv = ReplayDriver(ctx, shape, kv, pool_blocks, int(host_budget), wl.HASH_SEED, content, arena.alloc, lambda a: a,
-                       order="PF", log=log, free_pinned=arena.release, checkpoint="incremental")
+                       order="PF", log=log, free_pinned=arena.release, checkpoint="incremental", resident=(30, 131_072))
     streams, tg = {}, wl.rng(4, 2)
     checked_ckpt = checked_restore = 0
     try:
