@@ -159,15 +159,16 @@ def run_stage(torch, dev, ceilings, hbm_peak, reps=3) -> Dict:
         t_alone = _timed(torch, sa, lambda: ctx.stage(arr, bitmap, stream=sa), reps)
         prepared = ctx.stage_plan_create(arr)
         t_prepared = _timed(torch, sa, lambda: ctx.stage_plan_run(prepared, bitmap, stream=sa), reps)
-        t0 = time.perf_counter()
-        for _ in range(5):
-            ctx.stage_plan_run(prepared, bitmap, stream=sa)
-        host_us_prepared = (time.perf_counter() - t0) / 5 * 1e6
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(5):
-            ctx.stage(arr, bitmap, stream=sa)
-        host_us_plain = (time.perf_counter() - t0) / 5 * 1e6
+        def host_us(call):          # host time of one call, the GPU idle when it is made
+            ts = []
+            for _ in range(5):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                call()
+                ts.append(time.perf_counter() - t0)
+            return statistics.median(ts) * 1e6
+        host_us_prepared = host_us(lambda: ctx.stage_plan_run(prepared, bitmap, stream=sa))
+        host_us_plain = host_us(lambda: ctx.stage(arr, bitmap, stream=sa))
         torch.cuda.synchronize()
         ctx.stage_plan_destroy(prepared)
         t_res_alone = _timed(torch, sb, lambda: ctx.kv_restore(kv, table, 0, nblk, image, hl, stream=sb), reps)

@@ -114,6 +114,15 @@ bool RangeCache::covers(uintptr_t p, uintptr_t bytes) const {
   return p >= it->lo && p + bytes <= it->hi && p + bytes >= p;
 }
 
+bool RangeCache::find(uintptr_t p, AddrRange *out) const {
+  auto it = std::upper_bound(v.begin(), v.end(), p, [](uintptr_t x, const AddrRange &r) { return x < r.lo; });
+  if (it == v.begin()) return false;
+  --it;
+  if (p < it->lo || p >= it->hi) return false;
+  *out = *it;
+  return true;
+}
+
 void RangeCache::insert(AddrRange r) {
   // whatever overlaps the new range described memory that has been freed since
   v.erase(std::remove_if(v.begin(), v.end(), [&](const AddrRange &o) { return o.lo < r.hi && r.lo < o.hi; }), v.end());
@@ -169,6 +178,31 @@ talaria_status_t mapped_range(talaria_ctx *ctx, const void *host, int64_t bytes,
   void *last = nullptr;
   if (mapped_pointer(ctx, (const char *)host + (bytes - 1), &last) != TALARIA_OK) return TALARIA_ERR_EXTENT;
   return ((uintptr_t)last - (uintptr_t)*dev_alias == n - 1) ? TALARIA_OK : TALARIA_ERR_EXTENT;
+}
+
+talaria_status_t mapped_range(talaria_ctx *ctx, HostRangeMemo *memo, const void *host, int64_t bytes, void **dev_alias) {
+  const uintptr_t p = (uintptr_t)host;
+  if (bytes >= 0 && memo->alias_lo && p >= memo->lo && p + (uintptr_t)bytes >= p && p + (uintptr_t)bytes <= memo->hi) {
+    *dev_alias = (void *)(memo->alias_lo + (p - memo->lo));
+    return TALARIA_OK;
+  }
+  TAL_TRY(mapped_range(ctx, host, bytes, dev_alias));
+  // remember the registration or allocation that answered (the driver has just confirmed it)
+  AddrRange a{};
+  bool known = false;
+  for (const auto &r : ctx->registered)
+    if (p >= (uintptr_t)r.first && p < (uintptr_t)r.first + r.second) {
+      a = AddrRange{(uintptr_t)r.first, (uintptr_t)r.first + r.second};
+      known = true;
+      break;
+    }
+  if (!known) known = ctx->host_ranges.find(p, &a);
+  if (known) {
+    memo->lo = a.lo;
+    memo->hi = a.hi;
+    memo->alias_lo = (const char *)*dev_alias - (p - a.lo);
+  }
+  return TALARIA_OK;
 }
 
 talaria_status_t require_device_range(talaria_ctx *ctx, const void *ptr, int64_t bytes) {

@@ -45,6 +45,7 @@ struct AddrRange {
 struct RangeCache {
   std::vector<AddrRange> v;
   bool covers(uintptr_t p, uintptr_t bytes) const;
+  bool find(uintptr_t p, AddrRange *out) const;      // the cached range that holds p
   void insert(AddrRange r);
 };
 
@@ -150,6 +151,15 @@ talaria_status_t require_device_pointer(talaria_ctx *ctx, const void *p);
 // byte is wrong, EXTENT when the range runs off its allocation or registration.  With
 // validation off only the first byte is looked at.
 talaria_status_t mapped_range(talaria_ctx *ctx, const void *host, int64_t bytes, void **dev_alias);
+// The same for many ranges checked within ONE call: the pinned allocation that held the last
+// range is remembered together with its device alias, and later ranges inside it are answered
+// without asking the driver again (a plan with thousands of host-sourced chunks of one pinned
+// buffer would otherwise pay a driver query each).  A memo must not outlive the call.
+struct HostRangeMemo {
+  uintptr_t lo = 0, hi = 0;
+  const char *alias_lo = nullptr;
+};
+talaria_status_t mapped_range(talaria_ctx *ctx, HostRangeMemo *memo, const void *host, int64_t bytes, void **dev_alias);
 talaria_status_t require_device_range(talaria_ctx *ctx, const void *p, int64_t bytes);
 
 #ifdef __CUDACC__

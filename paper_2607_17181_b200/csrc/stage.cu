@@ -276,6 +276,7 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
   // ---- H2D leg, part 1: merge neighbouring host-sourced chunks and check every host
   // source before anything is enqueued, so a rejected plan leaves no partial copy behind.
   std::vector<LegItem> runs;
+  HostRangeMemo host_memo;
   for (int64_t k = 0; k < n;) {
     if (!from_host[(size_t)k] || plan[k].bytes == 0) { ++k; continue; }
     LegItem r{nullptr, (const char *)plan[k].src_host, (char *)plan[k].dst_dev, plan[k].bytes};
@@ -286,7 +287,7 @@ static talaria_status_t stage_impl(talaria_ctx *ctx, const talaria_copy_t *plan,
       ++j;
     }
     void *alias;
-    TAL_TRY(mapped_range(ctx, r.src_host, r.bytes, &alias));
+    TAL_TRY(mapped_range(ctx, &host_memo, r.src_host, r.bytes, &alias));
     r.src = (const char *)alias;               // kept beside the host address: the kernel leg reads through it
     runs.push_back(r);
     k = j;
@@ -376,11 +377,12 @@ static talaria_status_t plan_create(talaria_ctx *ctx, const talaria_copy_t *plan
     sp->plan.assign(plan, plan + n);
     sp->host_pinned.assign((size_t)n, 0);
     sp->host_alias.assign((size_t)n, nullptr);
+    HostRangeMemo host_memo;
     for (int64_t k = 0; k < n; ++k) {
       sp->tiles += (plan[k].bytes + kStageTile - 1) / kStageTile;
       if (plan[k].chunk_id > sp->max_chunk) sp->max_chunk = plan[k].chunk_id;
       void *alias = nullptr;
-      if (plan[k].src_host && mapped_range(ctx, plan[k].src_host, plan[k].bytes, &alias) == TALARIA_OK) {
+      if (plan[k].src_host && mapped_range(ctx, &host_memo, plan[k].src_host, plan[k].bytes, &alias) == TALARIA_OK) {
         sp->host_pinned[(size_t)k] = 1;
         sp->host_alias[(size_t)k] = (const char *)alias;
       }
@@ -531,9 +533,10 @@ static talaria_status_t prestage_impl(talaria_ctx *ctx, const talaria_copy_t *pl
       runs.push_back(HostRun{h, d, c.bytes});
     }
   }
+  HostRangeMemo host_memo;
   for (const HostRun &r : runs) {          // every range is checked before anything is enqueued
     void *alias;
-    TAL_TRY(mapped_range(ctx, r.h, r.bytes, &alias));
+    TAL_TRY(mapped_range(ctx, &host_memo, r.h, r.bytes, &alias));
     TAL_TRY(require_device_range(ctx, r.d, r.bytes));
   }
   for (const HostRun &r : runs) {
