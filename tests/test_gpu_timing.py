@@ -68,7 +68,7 @@ def test_timing_of_offload_restore_and_stage_legs():
         out_h = np.zeros(5200 // 16, np.uint64)
         ctx.prefix_match_host(1, cont, [0, cont.size], sess, [0, sess.size], None, 16, wl.HASH_SEED, out_h, res)
         t = ctx.get_timing()
-        assert t.op == 4 and 0 < t.total_ms < 50 and t.d2d_ms == 0 and t.h2d_ms == 0 and t.d2h_ms == 0
+        assert t.op == 4 and 0 < t.total_ms < 5000 and t.d2d_ms == 0 and t.h2d_ms == 0 and t.d2h_ms == 0
         d_tokens = torch.zeros(16384, dtype=torch.int32, device="cuda")
         d_hashes = torch.zeros(1024, dtype=torch.int64, device="cuda")
         ctx.stage(plan, None)
@@ -76,7 +76,7 @@ def test_timing_of_offload_restore_and_stage_legs():
         assert ctx.get_timing().op == 4
         ctx.prefix_match_resident([(cont, 8192, 512, 0, sess.size, 0)], d_tokens, d_hashes, 16, wl.HASH_SEED, res)
         t = ctx.get_timing()
-        assert t.op == 4 and 0 < t.total_ms < 50 and int(res[0]["lcp_tokens"]) == 4000
+        assert t.op == 4 and 0 < t.total_ms < 5000 and int(res[0]["lcp_tokens"]) == 4000
         ctx.set_timing(False)
         ctx.kv_offload(pool.kv, table, 0, 2, img.ptr, hl)
         ctx.sync()
