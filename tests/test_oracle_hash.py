@@ -133,6 +133,44 @@ def test_position_weights_never_alias_for_32bit_tokens():
         assert min(d, (1 << 64) - d) > (1 << 32)
 
 
+def test_finaliser_is_a_bijection_so_equal_hashes_mean_equal_chain_states():
+    # The block hash is the finaliser applied to the chain state.  Its inverse exists (undo the
+    # xor-shifts, multiply by the inverses of the two odd constants), so two block hashes are equal
+    # exactly when the chain states are -- which lets an implementation compare states, and lets it
+    # skip hashing a stored stream over the prefix where the tokens are equal.
+    def unshift(z, s):
+        x = z
+        for _ in range(64 // s + 1):
+            x = z ^ (x >> s)
+        return x
+
+    inv1, inv2 = pow(0xBF58476D1CE4E5B9, -1, 1 << 64), pow(0x94D049BB133111EB, -1, 1 << 64)
+
+    def unmix(h):
+        z = unshift(h, 31)
+        z = (z * inv2) & M64
+        z = unshift(z, 27)
+        z = (z * inv1) & M64
+        return unshift(z, 30)
+
+    g = wl.rng(77)
+    for x in [0, 1, M64, 1 << 63] + [int(v) for v in g.integers(0, 1 << 63, size=2000, dtype=np.int64)]:
+        assert unmix(orc.mix64(x)) == x
+    # and at the level of the chain: streams equal up to a block give equal hashes up to that block,
+    # and from the first different block on the hashes differ exactly where the states do
+    B, seed = 16, 0x54414C41524941
+    a = wl.tokens(g, 40 * B)
+    b = a.copy()
+    b[17 * B + 5] ^= 1
+    ha, hb = orc.block_hash(a, B, seed), orc.block_hash(b, B, seed)
+    assert np.array_equal(ha[:17], hb[:17]) and not np.any(ha[17:] == hb[17:])
+    sa, sb = seed, seed
+    for k in range(40):
+        sa = (sa * P + orc.block_digest(a[k * B:(k + 1) * B])) & M64
+        sb = (sb * P + orc.block_digest(b[k * B:(k + 1) * B])) & M64
+        assert (sa == sb) == (int(ha[k]) == int(hb[k]))
+
+
 def test_golden_config1_hashes():
     path = os.path.join(GOLDEN, "config1_hashes.txt")
     want = [int(ln, 16) for ln in open(path).read().splitlines() if ln.strip() and not ln.startswith("#")]
