@@ -89,7 +89,7 @@ def test_random_batches_mix_fused_and_single_transfers(case):
     g = wl.rng(1001, case)
     shape = wl.KvShape(int(g.integers(1, 5)), int(g.choice([1, 2])), 16, int(g.choice([8, 64])),
                        elt_bytes=int(g.choice([1, 2])), num_planes=int(g.choice([1, 2])))
-    nb = 400
+    nb = 640                                      # room for the largest draw: 13 sessions x 23 blocks, twice
     planes = [g.integers(0, 256, size=nb * shape.chunk_bytes, dtype=np.uint8)
               for _ in range(shape.num_layers * shape.num_planes)]
     pool = DevicePool(shape, planes)
