@@ -112,6 +112,36 @@ def test_many_sessions_in_one_call(n):
         ctx.destroy()
 
 
+@pytest.mark.parametrize("case", range(24))
+def test_random_sessions(case):
+    """Random block size (powers of two and others), number of sessions (every kernel route), stream
+    lengths including empty ones, alignment of the places, stored or derived hashes."""
+    g = wl.rng(1206, case)
+    B = int(g.choice([1, 3, 4, 8, 16, 24, 32, 64]))
+    n = int(g.choice([1, 2, 5, 8, 9, 20, 150, 200]))
+    longest = int(g.choice([200, 3000, 40000])) if n < 50 else int(g.choice([200, 3000]))
+    derive = bool(g.uniform() < 0.4)
+    ctx = tb.Talaria(0, host_match_bytes=2 << 20)
+    try:
+        arena = Arena(n, longest, B, odd=int(g.integers(0, 4)))
+        for turn in range(3):
+            conts = []
+            for s in range(n):
+                prev = arena.stored[s]
+                T = int(g.integers(0, longest + 1)) if g.uniform() < 0.9 else 0
+                shared = int(g.integers(0, min(prev.size, T) + 1)) if g.uniform() < 0.8 else min(prev.size, T)
+                conts.append(wl.continuation(g, prev, T, shared) if prev.size else wl.tokens(g, T))
+            res = np.zeros(n, tb.MATCH_DTYPE)
+            ctx.prefix_match_resident([arena.pair(s, conts[s], derive) for s in range(n)], arena.d_tokens, arena.d_hashes,
+                                      B, SEED, res)
+            for s in range(n):
+                _expect(res, s, conts[s], arena.stored[s], B, SEED)
+                arena.commit(s, conts[s], SEED)
+            arena.check()
+    finally:
+        ctx.destroy()
+
+
 def test_prompts_larger_than_the_staging_go_in_several_rounds():
     g = wl.rng(1203)
     B = 16
