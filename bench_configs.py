@@ -454,6 +454,53 @@ def run_sweep(torch, dev, ceilings) -> Dict:
             "value": max(b["offload_gbs"] for b in bounce)}
 
 
+def _match_from_host(torch, dev, ctx, g, n=4, T=36_000, B=16, reps=100) -> Dict:
+    """A returning group of n sessions, prompts in pageable host memory, on an idle link: every stream
+    sent up with the call (`prefix_match_host`) against streams and hashes kept on the device
+    (`prefix_match_resident`).  Host wall time per synchronous call, median."""
+    stored = [wl.tokens(g, T) for _ in range(n)]
+    conts = [wl.continuation(g, s, T + 2000, T - 1000) for s in stored]
+    want = [(T - 1000, (T - 1000) // B, (T - 1000) // B * B)] * n
+    res = np.zeros(n, tb.MATCH_DTYPE)
+    got = lambda: [(int(r["lcp_tokens"]), int(r["matched_blocks"]), int(r["reusable_tokens"])) for r in res]
+    # (a) everything from host memory
+    cont_all, sess_all = np.concatenate(conts), np.concatenate(stored)
+    co = np.cumsum([0] + [c.size for c in conts]).astype(np.int64)
+    so = np.cumsum([0] + [s.size for s in stored]).astype(np.int64)
+    hs = np.zeros(int(sum(s.size // B for s in stored)), np.uint64)
+    ctx.prefix_match_host(n, sess_all, so, sess_all, so, None, B, wl.HASH_SEED, hs, res)     # the stored streams' hashes
+    out_h = np.zeros(int(sum(c.size // B for c in conts)), np.uint64)
+    def timed(call):
+        ts = []
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            call()
+            ts.append(time.perf_counter() - t0)
+        return statistics.median(ts) * 1e6
+    us_host = timed(lambda: ctx.prefix_match_host(n, cont_all, co, sess_all, so, hs, B, wl.HASH_SEED, out_h, res))
+    ok = got() == want
+    # (b) stored streams and hashes resident: two places per session, used in turn
+    stride, hstride = 131_072, 131_072 // B
+    d_tokens = torch.zeros(2 * n * stride, dtype=torch.int32, device=dev)
+    d_hashes = torch.zeros(2 * n * hstride, dtype=torch.int64, device=dev)
+    ctx.prefix_match_resident([(stored[s], 2 * s * stride, 2 * s * hstride, (2 * s + 1) * stride, 0, -1) for s in range(n)],
+                              d_tokens, d_hashes, B, wl.HASH_SEED, res)
+    pairs = [(conts[s], (2 * s + 1) * stride, (2 * s + 1) * hstride, 2 * s * stride, stored[s].size, 2 * s * hstride)
+             for s in range(n)]
+    us_res = timed(lambda: ctx.prefix_match_resident(pairs, d_tokens, d_hashes, B, wl.HASH_SEED, res))
+    ok = ok and got() == want
+    ctx.set_timing(True)
+    ctx.prefix_match_resident(pairs, d_tokens, d_hashes, B, wl.HASH_SEED, res)
+    gpu_us = ctx.get_timing().total_ms * 1e3
+    ctx.set_timing(False)
+    same = bool(np.array_equal(d_hashes[(2 * 0 + 1) * hstride:(2 * 0 + 1) * hstride + conts[0].size // B].cpu().numpy().view(np.uint64),
+                               out_h[:conts[0].size // B]))
+    return {"sessions": n, "prompt_tokens": T + 2000, "stored_tokens": T,
+            "us_per_call_every_stream_from_host": us_host, "us_per_call_streams_resident": us_res,
+            "of_which_on_the_gpu_us_resident": gpu_us, "bytes_up_from_host": int(cont_all.nbytes + sess_all.nbytes + hs.nbytes),
+            "bytes_up_resident": int(cont_all.nbytes), "self_check": bool(ok and same)}
+
+
 def run_prefix(torch, dev, hbm_peak=6542.4, small=False) -> Dict:
     """Prefix-match latency for one returning session and throughput for a large batch.
     small: only the batch, cut to 444 pairs (one wave of the one-CTA-per-pair kernel, 155 MB of
@@ -483,6 +530,8 @@ def run_prefix(torch, dev, hbm_peak=6542.4, small=False) -> Dict:
                                   "us_per_call_gpu_back_to_back": back * 1e3, "us_call_plus_sync_via_python": lat * 1e6,
                                   "tokens_per_s_gpu": (Tc + Ts) / back * 1e3,
                                   "self_check": [int(r[0]), int(r[1]), int(r[2])] == [shared, shared // 16, shared // 16 * 16]})
+    if not small:
+        out["from_host"] = _match_from_host(torch, dev, ctx, g)
     npairs, T = (444 if small else 1024), 32768
     big_c = torch.randint(0, wl.VOCAB, (npairs * T,), dtype=torch.int32, device=dev)
     big_s = big_c.clone()
@@ -518,7 +567,7 @@ def run_prefix(torch, dev, hbm_peak=6542.4, small=False) -> Dict:
                              "frac_of_hbm_peak": 2 * npairs * T * 4 / ms / 1e6 / hbm_peak,
                              "mixes_per_s": mixes / ms * 1e3,
                              "frac_of_alu_ceiling_1.08e12_mixes_per_s": mixes / ms * 1e3 / 1.08e12})
-    out["self_check"] = ok
+    out["self_check"] = ok and out.get("from_host", {}).get("self_check", True)
     ctx.destroy()
     out["value"] = out["batch"][0]["tokens_per_s"]
     return out
