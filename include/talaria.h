@@ -231,8 +231,10 @@ talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t n_pairs,
  * (TALARIA_ERR_EXTENT; the arrays themselves inside their device allocations); no prompt or hash
  * destination overlaps another one or a stored range this call reads (TALARIA_ERR_OVERLAP).
  * A prompt larger than the staging (host_match_bytes) is TALARIA_ERR_EXTENT; a batch larger than
- * it runs as sub-batches of whole pairs.  Nothing is allocated.  Synchronous: returns after the
- * records are in h_results. */
+ * it runs as sub-batches of whole pairs.  Nothing is allocated.  Returns after the records are in
+ * h_results and the hashes in d_hashes; the prompts reach their places in d_tokens in stream order
+ * (work enqueued on `stream` afterwards sees them; another stream must be ordered after `stream`
+ * first, e.g. by talaria_sync). */
 typedef struct {
   const int32_t *h_cont_tokens;   /* HOST [cont_tokens] */
   int64_t cont_tokens;

@@ -242,6 +242,8 @@ static void destroy_impl(talaria_ctx *ctx) {
   }
   for (cudaEvent_t e : ctx->tm)
     if (e) cudaEventDestroy(e);
+  if (ctx->match_done) cudaEventDestroy(ctx->match_done);
+  if (ctx->stage_free) cudaEventDestroy(ctx->stage_free);
   if (ctx->reload_fork) cudaEventDestroy(ctx->reload_fork);
   if (ctx->reload_done) cudaEventDestroy(ctx->reload_done);
   for (auto &s : ctx->ring) {
@@ -308,6 +310,8 @@ extern "C" talaria_status_t talaria_create(talaria_ctx **out, int32_t device, co
     TAL_TRY(grow(ctx, &ctx->host_tok, (size_t)ctx->cfg.host_match_bytes));
     TAL_CUDA(ctx, cudaHostAlloc((void **)&ctx->match_pin, ctx->host_tok.cap, cudaHostAllocMapped));
     TAL_CUDA(ctx, cudaHostGetDevicePointer((void **)&ctx->match_pin_dev, ctx->match_pin, 0));
+    TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->match_done, cudaEventDisableTiming));
+    TAL_CUDA(ctx, cudaEventCreateWithFlags(&ctx->stage_free, cudaEventDisableTiming));
     // Internal streams run at the highest priority: their kernels are short packing
     // steps that gate copy-engine transfers, so they should not queue behind a long
     // kernel of the caller's (for example a staging copy on another stream).

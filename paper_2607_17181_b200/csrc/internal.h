@@ -71,6 +71,10 @@ struct talaria_ctx {
   cudaStream_t prefix_stream = nullptr;  // stream of that call (same stream: already ordered)
   tal::DevBuf host_tok;               // device side of talaria_prefix_match_host's staging (fixed size)
   char *match_pin = nullptr;          // pinned side, same size and layout
+  cudaEvent_t match_done = nullptr;   // resident match: its kernels have written the result records
+  cudaEvent_t stage_free = nullptr;   // ... and the prompts have been spread out of the device staging
+  bool stage_busy = false;            // a spread may still be reading the device staging
+  cudaStream_t stage_stream = nullptr;  // ... on this stream
   char *match_pin_dev = nullptr;      // ... as the device sees it (results are written through this mapping)
   std::vector<std::pair<char *, size_t>> registered;
   tal::RangeCache host_ranges;        // pinned host allocations seen so far

@@ -597,6 +597,8 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
   auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
   const size_t cap = ctx->host_tok.cap;
   char *const dev = ctx->host_tok.p, *const pin = ctx->match_pin;
+  // a resident match on another stream may still be spreading prompts out of the device staging
+  if (ctx->stage_busy && ctx->stage_stream != stream) TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->stage_free, 0));
   std::vector<int64_t> co, so;
   int64_t sb_before = 0, cb_before = 0;           // blocks of the pairs already done (positions in the users' hash arrays)
   for (int32_t q0 = 0; q0 < n_pairs;) {
@@ -655,6 +657,26 @@ extern "C" talaria_status_t talaria_prefix_match_host(talaria_ctx *ctx, int32_t 
   return TALARIA_OK;
 }
 
+
+namespace tal {
+
+// Prompts out of the device staging into their places in the caller's token array.
+constexpr int kSpreadItems = 64;
+struct SpreadParams {
+  const int32_t *src;
+  int32_t *dst;
+  int32_t n;
+  int64_t src_off[kSpreadItems], dst_off[kSpreadItems], count[kSpreadItems];   // in elements
+};
+__global__ void __launch_bounds__(256) resident_spread_kernel(const __grid_constant__ SpreadParams p) {
+  const int it = blockIdx.y;
+  const int32_t *src = p.src + p.src_off[it];
+  int32_t *dst = p.dst + p.dst_off[it];
+  const int64_t n = p.count[it], step = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += step) dst[i] = __ldg(src + i);
+}
+
+}  // namespace tal
 
 // Match against streams that live on the device (Sec. 4.3: the instance keeps what it knows of a
 // session; App. A: the new prompt is compared with it).  Only the new prompt crosses the host
@@ -717,6 +739,7 @@ extern "C" talaria_status_t talaria_prefix_match_resident(talaria_ctx *ctx, int3
   const size_t cap = ctx->host_tok.cap;
   char *const pin = ctx->match_pin, *const pin_dev = ctx->match_pin_dev;
   std::vector<PairSpec> specs;
+  if (ctx->stage_busy && ctx->stage_stream != stream) TAL_CUDA(ctx, cudaStreamWaitEvent(stream, ctx->stage_free, 0));
   for (int32_t q0 = 0; q0 < n_pairs;) {
     // the longest run of whole pairs whose prompts and result records fit the pinned staging
     int32_t q1 = q0;
@@ -731,19 +754,23 @@ extern "C" talaria_status_t talaria_prefix_match_resident(talaria_ctx *ctx, int3
     const int32_t m = q1 - q0;
     const size_t o_res = bytes;
     specs.resize((size_t)m);
-    // The prompts are packed in the pinned staging, cross the host link in ONE copy (a copy per
-    // prompt pays the link's latency once each, and several times over while checkpoints keep the
-    // other direction busy), and are spread to their places by device-to-device copies.
+    // Every command the GPU fetches costs a round trip on the host link, and several times that
+    // while a checkpoint keeps the link's other direction full (measured: +40 to +65 us per copy
+    // or launch).  So the call's critical path is two commands: ONE copy takes the packed prompts
+    // to the device staging and the match kernels read them there.  Spreading them to their places
+    // in the caller's array comes after the kernels and is not waited for.
     size_t at = 0;
+    int32_t n_spread = 0;
     for (int32_t q = q0; q < q1; ++q) {
       const talaria_resident_pair_t &r = pairs[q];
+      specs[(size_t)(q - q0)] = PairSpec{(int64_t)(at / 4), r.cont_tokens, r.sess_tokens > 0 ? r.sess_slot : 0, r.sess_tokens,
+                                         r.cont_tokens / B > 0 ? r.cont_hash_slot : 0,
+                                         (any_stored && r.sess_tokens / B > 0) ? r.sess_hash_slot : 0};
       if (r.cont_tokens > 0) {
         memcpy(pin + at, r.h_cont_tokens, (size_t)r.cont_tokens * 4);
         at += up((size_t)r.cont_tokens * 4);
+        ++n_spread;
       }
-      specs[(size_t)(q - q0)] = PairSpec{r.cont_slot, r.cont_tokens, r.sess_tokens > 0 ? r.sess_slot : 0, r.sess_tokens,
-                                         r.cont_tokens / B > 0 ? r.cont_hash_slot : 0,
-                                         (any_stored && r.sess_tokens / B > 0) ? r.sess_hash_slot : 0};
     }
     if (ctx->timing && q0 == 0) {      // op 4: from the first copy to the last kernel, host-side packing excluded
       ctx->tm_op = 4;
@@ -753,20 +780,37 @@ extern "C" talaria_status_t talaria_prefix_match_resident(talaria_ctx *ctx, int3
     if (at) {
       TAL_CUDA(ctx, cudaMemcpyAsync(ctx->host_tok.p, pin, at, cudaMemcpyHostToDevice, stream));
       ctx->counters.memcpy_calls++;
-      at = 0;
-      for (int32_t q = q0; q < q1; ++q) {
-        const talaria_resident_pair_t &r = pairs[q];
-        if (r.cont_tokens == 0) continue;
-        TAL_CUDA(ctx, cudaMemcpyAsync(d_tokens + r.cont_slot, ctx->host_tok.p + at, (size_t)r.cont_tokens * 4,
-                                      cudaMemcpyDeviceToDevice, stream));
-        ctx->counters.memcpy_calls++;
-        at += up((size_t)r.cont_tokens * 4);
-      }
     }
-    TAL_TRY(prefix_launch_specs(ctx, m, specs.data(), d_tokens, d_tokens, any_stored ? d_hashes : nullptr, B, seed,
-                                d_hashes, (talaria_match_t *)(pin_dev + o_res), stream));
+    TAL_TRY(prefix_launch_specs(ctx, m, specs.data(), (const int32_t *)ctx->host_tok.p, d_tokens,
+                                any_stored ? d_hashes : nullptr, B, seed, d_hashes,
+                                (talaria_match_t *)(pin_dev + o_res), stream));
     if (ctx->timing) TAL_CUDA(ctx, cudaEventRecord(ctx->tm[1], stream));
-    TAL_CUDA(ctx, cudaStreamSynchronize(stream));
+    TAL_CUDA(ctx, cudaEventRecord(ctx->match_done, stream));
+    for (int32_t q = q0; q < q1 && n_spread > 0;) {
+      SpreadParams sp{};
+      sp.src = (const int32_t *)ctx->host_tok.p;
+      sp.dst = d_tokens;
+      int64_t longest = 0;
+      for (; q < q1 && sp.n < kSpreadItems; ++q) {
+        if (pairs[q].cont_tokens == 0) continue;
+        sp.src_off[sp.n] = specs[(size_t)(q - q0)].cont_off;
+        sp.dst_off[sp.n] = pairs[q].cont_slot;
+        sp.count[sp.n] = pairs[q].cont_tokens;
+        longest = std::max(longest, pairs[q].cont_tokens);
+        ++sp.n;
+      }
+      if (sp.n == 0) break;
+      const unsigned gx = (unsigned)std::min<int64_t>((longest + 1023) / 1024, 64);
+      resident_spread_kernel<<<dim3(gx, (unsigned)sp.n), 256, 0, stream>>>(sp);
+      TAL_CUDA(ctx, cudaGetLastError());
+      ctx->counters.kernel_launches++;
+    }
+    TAL_CUDA(ctx, cudaEventRecord(ctx->stage_free, stream));
+    ctx->stage_busy = true;
+    ctx->stage_stream = stream;
+    // the records are complete once the match kernels are; a further round reuses the pinned
+    // staging, whose copy to the device precedes those kernels
+    TAL_CUDA(ctx, cudaEventSynchronize(ctx->match_done));
     memcpy(h_results + q0, pin + o_res, (size_t)m * sizeof(talaria_match_t));
     q0 = q1;
   }
